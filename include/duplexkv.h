@@ -1,0 +1,192 @@
+/*
+ * duplexkv.h -- C ABI of the B200 KV-block rotation engine.
+ *
+ * The operations are the data movement that the paper's DuplexKV rotation engine performs
+ * (section 4.3, "Efficient Offloading and Memory Management"): a request's paged KV cache is
+ * a set of fixed-size blocks scattered over a pool; rotating requests means copying the blocks
+ * of some requests from GPU HBM to host DRAM (swap-out) and the blocks of others from host
+ * DRAM into newly allocated HBM blocks (swap-in), with both directions in flight at once so
+ * that the host link is used full-duplex.
+ *
+ * Layouts (elements are 16-bit words, never interpreted):
+ *   device pool   [layer][K|V][block][block_size][kv_heads][head_dim]      ("layer-first")
+ *   host pool     [block][layer][K|V][block_size][kv_heads][head_dim]      ("block-first", default;
+ *                 the paper's merged layout: all layers of one block contiguous), or layer-first
+ *                 like the device pool.
+ * SEG  = block_size*kv_heads*head_dim*2 bytes: one K or V plane of one block in one layer, the
+ *        largest contiguous unit of the device layout.  SEG must be a multiple of 16.
+ * BLK  = 2*num_layers*SEG bytes: one block over all layers.
+ * Device byte offset of plane (l,kv) of block b: ((l*2+kv)*num_gpu_blocks + b)*SEG.
+ * Host byte offset (block-first) of plane (l,kv) of block h: h*BLK + (l*2+kv)*SEG.
+ *
+ * Conventions
+ *   - Every function returns a status (0 = KV_OK, negative = error); none throws, aborts or prints.
+ *   - Id arrays are HOST pointers to int32 block ids; they are copied during the call.
+ *   - Data-moving calls are asynchronous with respect to the device.  Swap-outs run in issue order on
+ *     the pool's "out" stream, swap-ins on its "in" stream; a call is ordered after an earlier call of
+ *     the other direction only when their lists touch the same block.  kv_sync waits for everything.
+ *   - On any validation error nothing is launched and no byte moves.
+ *   - One caller thread per pool.  There is no CPU fallback: every call needs the CUDA device.
+ */
+#ifndef DUPLEXKV_H_
+#define DUPLEXKV_H_
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+/* status codes */
+#define KV_OK                 0
+#define KV_ERR_INVALID_ARG   (-1)   /* null pointer, negative count, bad shape, count beyond pool size   */
+#define KV_ERR_RANGE         (-2)   /* a block id outside [0, num_blocks) of its pool                    */
+#define KV_ERR_DUP_DST       (-3)   /* the same destination block twice in one direction of one call     */
+#define KV_ERR_HAZARD        (-4)   /* rotate lists overlap across directions and overlap is not allowed */
+#define KV_ERR_CUDA          (-5)   /* a CUDA call failed; kv_last_error has the text                    */
+#define KV_ERR_TIMEOUT       (-6)   /* a bounded device-side wait ran out (reported by kv_sync)          */
+#define KV_ERR_NOMEM         (-7)   /* host or device allocation failed                                  */
+#define KV_ERR_UNSUPPORTED   (-8)   /* combination not provided (e.g. SEG not a multiple of 16)          */
+
+/* host pool layout */
+#define KV_HOST_BLOCK_FIRST   0
+#define KV_HOST_LAYER_FIRST   1
+
+/* transfer paths (how the host link is driven) */
+#define KV_PATH_AUTO          0     /* per-block-size choice measured on B200 (see kv_path_for)          */
+#define KV_PATH_ZEROCOPY      1     /* SM kernels read/write mapped pinned host memory directly          */
+#define KV_PATH_STAGED        2     /* pack kernel -> contiguous HBM staging -> copy engine (and reverse)*/
+#define KV_PATH_CE2D          3     /* one strided 2-D copy-engine transfer per block, no kernel         */
+#define KV_PATH_NAIVE         4     /* one copy-engine transfer per segment (the paper's "Naive" row)    */
+
+/* flags */
+#define KV_FLAG_ALLOW_OVERLAP   1   /* kv_rotate accepts lists that overlap across directions and orders
+                                       the conflicting swap-ins after the swap-out                       */
+#define KV_FLAG_LDST_KERNEL     2   /* ZEROCOPY/STAGED kernels use plain 16-byte loads/stores instead of
+                                       bulk asynchronous copies through shared memory                    */
+#define KV_FLAG_FUSED_ROTATE    4   /* ZEROCOPY kv_rotate with disjoint lists: one launch, CTAs split
+                                       between the directions, on the out stream                         */
+
+typedef struct kv_pool kv_pool_t;   /* opaque; owned by the library */
+
+typedef struct {
+    int32_t num_layers, block_size, kv_heads, head_dim;   /* element = 2 bytes, fixed                     */
+    int64_t num_gpu_blocks, num_host_blocks;
+    void   *device_base;    /* DEVICE pointer, required: >= num_gpu_blocks*BLK bytes, 256-byte aligned;
+                               borrowed (typically a torch tensor's storage)                              */
+    void   *host_base;      /* HOST pointer or NULL.  NULL: the library allocates num_host_blocks*BLK
+                               bytes of mapped pinned memory and owns it.  Non-NULL: caller memory of that
+                               size, 4096-byte aligned; the library page-locks it for the pool's lifetime */
+    int32_t host_layout;    /* KV_HOST_BLOCK_FIRST or KV_HOST_LAYER_FIRST                                 */
+    int32_t device_id;
+    void   *stream_out;     /* cudaStream_t or NULL (library creates a non-blocking stream)               */
+    void   *stream_in;      /* likewise; must differ from stream_out for the directions to overlap        */
+    int32_t path;           /* KV_PATH_*                                                                  */
+    int32_t flags;          /* KV_FLAG_*                                                                  */
+    int32_t ctas_out;       /* CTAs of the swap-out kernel, 0 = default for the path                      */
+    int32_t ctas_in;        /* CTAs of the swap-in kernel, 0 = default                                    */
+    int64_t staging_bytes;  /* per-direction HBM staging buffer of the STAGED path, 0 = 64 MiB            */
+} kv_pool_config_t;
+
+typedef struct {
+    int64_t bytes_out, bytes_in;       /* payload bytes moved since the pool was created                  */
+    int64_t calls_out, calls_in;       /* data-moving calls per direction                                 */
+    int64_t kernel_launches;           /* kernels this library launched                                   */
+    int64_t ce_copies;                 /* copy-engine transfers this library issued                       */
+    double  last_out_ms, last_in_ms;   /* device time of the latest completed call per direction,
+                                          from events on the launching streams; valid after kv_sync       */
+    double  last_union_ms;             /* first start to last end of the latest call (both directions
+                                          for kv_rotate)                                                  */
+    int32_t last_path_out, last_path_in;
+    uint32_t device_status;            /* sticky bits written by kernels (0 = clean)                      */
+    int32_t pad_;
+} kv_stats_t;
+
+typedef struct {
+    double d2h_gbs, h2d_gbs;           /* each direction alone, GB/s (1e9 bytes per second)               */
+    double bi_d2h_gbs, bi_h2d_gbs;     /* both at once: per-direction rates over the common window        */
+    double bi_sum_gbs;                 /* both at once: total bytes / window                              */
+    int64_t bytes; int32_t reps, pad_;
+} kv_link_probe_t;
+
+/*
+ * Create a pool descriptor over caller device memory and (owned or borrowed) pinned host memory.
+ * Sets the current device to cfg->device_id.  *out is NULL on failure.
+ * Follows the paper's two-pool picture (HBM pool and DRAM swap space, section 5.1 set-up).
+ */
+int32_t kv_pool_create(const kv_pool_config_t *cfg, kv_pool_t **out);
+
+/* Waits for all outstanding work, then frees what the library owns (never device_base, never a
+ * caller-supplied host_base, never caller streams). */
+int32_t kv_pool_destroy(kv_pool_t *pool);
+
+/*
+ * Swap-out (section 4.3: copy every segment of each listed HBM block to its DRAM block).
+ * For i < n, every layer l and plane kv: host block host_ids[i] plane (l,kv) <- device block
+ * gpu_ids[i] plane (l,kv).  The device pool is not modified.  host_ids must be unique
+ * (KV_ERR_DUP_DST); gpu_ids may repeat.  n == 0 is a no-op.  Asynchronous.
+ */
+int32_t kv_swap_out(kv_pool_t *pool, const int32_t *gpu_ids, const int32_t *host_ids, int64_t n);
+
+/*
+ * Swap-in (section 4.3: copy every segment of each listed DRAM block into a newly allocated HBM
+ * block).  For j < n: device block gpu_ids[j] <- host block host_ids[j], all planes.  The host pool
+ * is not modified.  gpu_ids must be unique; host_ids may repeat.  Asynchronous.
+ */
+int32_t kv_swap_in(kv_pool_t *pool, const int32_t *host_ids, const int32_t *gpu_ids, int64_t n);
+
+/*
+ * Rotation: swap-out of (out_gpu -> out_host) and swap-in of (in_host -> in_gpu) in one call, both
+ * directions in flight together.  The result is defined as swap-out THEN swap-in.  When a swap-in
+ * destination is a swap-out source, or a swap-in source is a swap-out destination (the data race of
+ * the paper's eager-block-rotation discussion), the call fails with KV_ERR_HAZARD and moves nothing,
+ * unless the pool was created with KV_FLAG_ALLOW_OVERLAP: then the conflicting swap-in pairs are
+ * issued after the swap-out completes and the rest still overlap.  Asynchronous.
+ */
+int32_t kv_rotate(kv_pool_t *pool,
+                  const int32_t *out_gpu, const int32_t *out_host, int64_t n_out,
+                  const int32_t *in_host, const int32_t *in_gpu, int64_t n_in);
+
+/* Wait for both directions.  Returns KV_OK, or the first sticky asynchronous error
+ * (KV_ERR_CUDA, KV_ERR_TIMEOUT).  Fills the last_* timing fields of the statistics. */
+int32_t kv_sync(kv_pool_t *pool);
+
+/*
+ * Device-side gather / scatter (the kernel half of the STAGED path, also usable on its own):
+ * gather copies the listed device blocks, in list order, into a contiguous DEVICE buffer laid out
+ * block-first (block i at i*BLK, planes in (layer, K|V) order); scatter is the inverse.  dst/src must
+ * hold n*BLK bytes and be 16-byte aligned.  Runs on the out (gather) / in (scatter) stream.
+ * This is the "merge small segments into large contiguous regions" step of section 4.3, done by
+ * a kernel instead of a layout change.
+ */
+int32_t kv_gather_blocks(kv_pool_t *pool, const int32_t *gpu_ids, int64_t n, void *dst_device);
+int32_t kv_scatter_blocks(kv_pool_t *pool, const void *src_device, const int32_t *gpu_ids, int64_t n);
+
+/* Host pool base (HOST pointer) and size, for filling and verification. */
+int32_t kv_host_ptr(kv_pool_t *pool, void **base, int64_t *bytes);
+
+int32_t kv_get_stats(kv_pool_t *pool, kv_stats_t *stats);
+
+/* Text of the latest error on this pool (never NULL; static storage inside the pool).
+ * With pool == NULL: the text of the latest kv_pool_create / kv_probe_link failure. */
+const char *kv_last_error(kv_pool_t *pool);
+
+/* SEG and BLK for a shape (bytes); 0 if the shape is invalid. */
+int64_t kv_seg_bytes(int32_t block_size, int32_t kv_heads, int32_t head_dim);
+int64_t kv_blk_bytes(int32_t num_layers, int32_t block_size, int32_t kv_heads, int32_t head_dim);
+
+/* The path KV_PATH_AUTO resolves to for a segment size. */
+int32_t kv_path_for(int64_t seg_bytes);
+
+/*
+ * Host-link roofline probe (the analogue of the paper's appendix B bandwidth measurement, done
+ * with plain pinned copy-engine transfers): times `reps` copies of `bytes` device->host, host->device,
+ * and both at once on two streams; best of three rounds after one warm-up.  Allocates and frees
+ * its own pinned and device buffers.
+ */
+int32_t kv_probe_link(int32_t device_id, int64_t bytes, int32_t reps, kv_link_probe_t *out);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* DUPLEXKV_H_ */

@@ -1,0 +1,248 @@
+"""ctypes binding of ``libduplexkv.so``: argument marshalling only.
+
+Every function here has the name and the semantics of the C entry point it wraps (see
+``include/duplexkv.h``); all data movement happens inside the CUDA library.  If the library
+is missing it is built with nvcc; if that fails, importing raises: there is no fallback.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+from typing import Optional, Sequence
+
+import numpy as np
+
+from . import build as _build
+
+KV_OK = 0
+KV_ERR_INVALID_ARG = -1
+KV_ERR_RANGE = -2
+KV_ERR_DUP_DST = -3
+KV_ERR_HAZARD = -4
+KV_ERR_CUDA = -5
+KV_ERR_TIMEOUT = -6
+KV_ERR_NOMEM = -7
+KV_ERR_UNSUPPORTED = -8
+
+KV_HOST_BLOCK_FIRST = 0
+KV_HOST_LAYER_FIRST = 1
+
+KV_PATH_AUTO = 0
+KV_PATH_ZEROCOPY = 1
+KV_PATH_STAGED = 2
+KV_PATH_CE2D = 3
+KV_PATH_NAIVE = 4
+PATH_NAMES = {0: "auto", 1: "zerocopy", 2: "staged", 3: "ce2d", 4: "naive"}
+
+KV_FLAG_ALLOW_OVERLAP = 1
+KV_FLAG_LDST_KERNEL = 2
+KV_FLAG_FUSED_ROTATE = 4
+
+
+class kv_pool_config_t(C.Structure):
+    _fields_ = [("num_layers", C.c_int32), ("block_size", C.c_int32), ("kv_heads", C.c_int32),
+                ("head_dim", C.c_int32), ("num_gpu_blocks", C.c_int64), ("num_host_blocks", C.c_int64),
+                ("device_base", C.c_void_p), ("host_base", C.c_void_p), ("host_layout", C.c_int32),
+                ("device_id", C.c_int32), ("stream_out", C.c_void_p), ("stream_in", C.c_void_p),
+                ("path", C.c_int32), ("flags", C.c_int32), ("ctas_out", C.c_int32), ("ctas_in", C.c_int32),
+                ("staging_bytes", C.c_int64)]
+
+
+class kv_stats_t(C.Structure):
+    _fields_ = [("bytes_out", C.c_int64), ("bytes_in", C.c_int64), ("calls_out", C.c_int64),
+                ("calls_in", C.c_int64), ("kernel_launches", C.c_int64), ("ce_copies", C.c_int64),
+                ("last_out_ms", C.c_double), ("last_in_ms", C.c_double), ("last_union_ms", C.c_double),
+                ("last_path_out", C.c_int32), ("last_path_in", C.c_int32),
+                ("device_status", C.c_uint32), ("pad_", C.c_int32)]
+
+
+class kv_link_probe_t(C.Structure):
+    _fields_ = [("d2h_gbs", C.c_double), ("h2d_gbs", C.c_double), ("bi_d2h_gbs", C.c_double),
+                ("bi_h2d_gbs", C.c_double), ("bi_sum_gbs", C.c_double), ("bytes", C.c_int64),
+                ("reps", C.c_int32), ("pad_", C.c_int32)]
+
+
+EXPORTS = ["kv_pool_create", "kv_pool_destroy", "kv_swap_out", "kv_swap_in", "kv_rotate", "kv_sync",
+           "kv_gather_blocks", "kv_scatter_blocks", "kv_host_ptr", "kv_get_stats", "kv_last_error",
+           "kv_seg_bytes", "kv_blk_bytes", "kv_path_for", "kv_probe_link"]
+
+_lib = None
+
+
+def lib() -> C.CDLL:
+    """Load (building first if needed) the CUDA library.  Raises if it cannot be had."""
+    global _lib
+    if _lib is not None:
+        return _lib
+    path = _build.build()
+    L = C.CDLL(path)
+    i32p, vp, i64 = C.POINTER(C.c_int32), C.c_void_p, C.c_int64
+    L.kv_pool_create.restype = C.c_int32
+    L.kv_pool_create.argtypes = [C.POINTER(kv_pool_config_t), C.POINTER(vp)]
+    L.kv_pool_destroy.restype = C.c_int32
+    L.kv_pool_destroy.argtypes = [vp]
+    L.kv_swap_out.restype = C.c_int32
+    L.kv_swap_out.argtypes = [vp, i32p, i32p, i64]
+    L.kv_swap_in.restype = C.c_int32
+    L.kv_swap_in.argtypes = [vp, i32p, i32p, i64]
+    L.kv_rotate.restype = C.c_int32
+    L.kv_rotate.argtypes = [vp, i32p, i32p, i64, i32p, i32p, i64]
+    L.kv_sync.restype = C.c_int32
+    L.kv_sync.argtypes = [vp]
+    L.kv_gather_blocks.restype = C.c_int32
+    L.kv_gather_blocks.argtypes = [vp, i32p, i64, vp]
+    L.kv_scatter_blocks.restype = C.c_int32
+    L.kv_scatter_blocks.argtypes = [vp, vp, i32p, i64]
+    L.kv_host_ptr.restype = C.c_int32
+    L.kv_host_ptr.argtypes = [vp, C.POINTER(vp), C.POINTER(i64)]
+    L.kv_get_stats.restype = C.c_int32
+    L.kv_get_stats.argtypes = [vp, C.POINTER(kv_stats_t)]
+    L.kv_last_error.restype = C.c_char_p
+    L.kv_last_error.argtypes = [vp]
+    L.kv_seg_bytes.restype = i64
+    L.kv_seg_bytes.argtypes = [C.c_int32] * 3
+    L.kv_blk_bytes.restype = i64
+    L.kv_blk_bytes.argtypes = [C.c_int32] * 4
+    L.kv_path_for.restype = C.c_int32
+    L.kv_path_for.argtypes = [i64]
+    L.kv_probe_link.restype = C.c_int32
+    L.kv_probe_link.argtypes = [C.c_int32, i64, C.c_int32, C.POINTER(kv_link_probe_t)]
+    _lib = L
+    return L
+
+
+def lib_path() -> str:
+    return _build.LIB
+
+
+class KVError(RuntimeError):
+    def __init__(self, code: int, msg: str):
+        super().__init__(f"duplexkv error {code}: {msg}")
+        self.code = code
+
+
+def _ids(a) -> tuple:
+    arr = np.ascontiguousarray(np.asarray(a, dtype=np.int32))
+    return arr, arr.ctypes.data_as(C.POINTER(C.c_int32))
+
+
+def kv_seg_bytes(block_size: int, kv_heads: int, head_dim: int) -> int:
+    return lib().kv_seg_bytes(block_size, kv_heads, head_dim)
+
+
+def kv_blk_bytes(num_layers: int, block_size: int, kv_heads: int, head_dim: int) -> int:
+    return lib().kv_blk_bytes(num_layers, block_size, kv_heads, head_dim)
+
+
+def kv_path_for(seg_bytes: int) -> int:
+    return lib().kv_path_for(seg_bytes)
+
+
+def kv_probe_link(device_id: int = 0, nbytes: int = 256 << 20, reps: int = 4) -> dict:
+    out = kv_link_probe_t()
+    rc = lib().kv_probe_link(device_id, nbytes, reps, C.byref(out))
+    if rc != KV_OK:
+        raise KVError(rc, lib().kv_last_error(None).decode())
+    return {k: getattr(out, k) for k, _ in kv_link_probe_t._fields_ if k != "pad_"}
+
+
+class KVPool:
+    """Thin owner of a ``kv_pool_t*``.  Methods return the C status code unchanged unless
+    ``check=True`` (default), in which case a negative status raises ``KVError``."""
+
+    def __init__(self, num_layers: int, block_size: int, kv_heads: int, head_dim: int,
+                 num_gpu_blocks: int, num_host_blocks: int, device_base: int, *,
+                 host_base: Optional[int] = None, host_layout: int = KV_HOST_BLOCK_FIRST,
+                 device_id: int = 0, stream_out: Optional[int] = None, stream_in: Optional[int] = None,
+                 path: int = KV_PATH_AUTO, flags: int = 0, ctas_out: int = 0, ctas_in: int = 0,
+                 staging_bytes: int = 0):
+        self.cfg = kv_pool_config_t(num_layers, block_size, kv_heads, head_dim, num_gpu_blocks,
+                                    num_host_blocks, device_base, host_base, host_layout, device_id,
+                                    stream_out, stream_in, path, flags, ctas_out, ctas_in, staging_bytes)
+        self._h = C.c_void_p()
+        rc = lib().kv_pool_create(C.byref(self.cfg), C.byref(self._h))
+        if rc != KV_OK:
+            raise KVError(rc, lib().kv_last_error(None).decode())
+        self.seg = kv_seg_bytes(block_size, kv_heads, head_dim)
+        self.blk = kv_blk_bytes(num_layers, block_size, kv_heads, head_dim)
+
+    # -- lifetime
+    def destroy(self) -> None:
+        if self._h:
+            lib().kv_pool_destroy(self._h)
+            self._h = C.c_void_p()
+
+    def __del__(self):
+        try:
+            self.destroy()
+        except Exception:
+            pass
+
+    def __enter__(self):
+        return self
+
+    def __exit__(self, *exc):
+        self.destroy()
+
+    def _ret(self, rc: int, check: bool) -> int:
+        if check and rc != KV_OK:
+            raise KVError(rc, self.kv_last_error())
+        return rc
+
+    # -- the C entry points
+    def kv_swap_out(self, gpu_ids, host_ids, check: bool = True) -> int:
+        g, gp = _ids(gpu_ids)
+        h, hp = _ids(host_ids)
+        if len(g) != len(h):
+            raise ValueError("gpu_ids and host_ids differ in length")
+        return self._ret(lib().kv_swap_out(self._h, gp, hp, len(g)), check)
+
+    def kv_swap_in(self, host_ids, gpu_ids, check: bool = True) -> int:
+        h, hp = _ids(host_ids)
+        g, gp = _ids(gpu_ids)
+        if len(g) != len(h):
+            raise ValueError("gpu_ids and host_ids differ in length")
+        return self._ret(lib().kv_swap_in(self._h, hp, gp, len(g)), check)
+
+    def kv_rotate(self, out_gpu, out_host, in_host, in_gpu, check: bool = True) -> int:
+        og, ogp = _ids(out_gpu)
+        oh, ohp = _ids(out_host)
+        ih, ihp = _ids(in_host)
+        ig, igp = _ids(in_gpu)
+        if len(og) != len(oh) or len(ih) != len(ig):
+            raise ValueError("paired lists differ in length")
+        return self._ret(lib().kv_rotate(self._h, ogp, ohp, len(og), ihp, igp, len(ig)), check)
+
+    def kv_rotate_raw(self, ogp, ohp, n_out, ihp, igp, n_in) -> int:
+        """Same call with pre-marshalled ``POINTER(c_int32)`` arguments (for timing loops)."""
+        return lib().kv_rotate(self._h, ogp, ohp, n_out, ihp, igp, n_in)
+
+    def kv_sync(self, check: bool = True) -> int:
+        return self._ret(lib().kv_sync(self._h), check)
+
+    def kv_gather_blocks(self, gpu_ids, dst_device: int, check: bool = True) -> int:
+        g, gp = _ids(gpu_ids)
+        return self._ret(lib().kv_gather_blocks(self._h, gp, len(g), dst_device), check)
+
+    def kv_scatter_blocks(self, src_device: int, gpu_ids, check: bool = True) -> int:
+        g, gp = _ids(gpu_ids)
+        return self._ret(lib().kv_scatter_blocks(self._h, src_device, gp, len(g)), check)
+
+    def kv_host_ptr(self) -> tuple:
+        base, nbytes = C.c_void_p(), C.c_int64()
+        self._ret(lib().kv_host_ptr(self._h, C.byref(base), C.byref(nbytes)), True)
+        return base.value, nbytes.value
+
+    def kv_get_stats(self) -> dict:
+        st = kv_stats_t()
+        self._ret(lib().kv_get_stats(self._h, C.byref(st)), True)
+        return {k: getattr(st, k) for k, _ in kv_stats_t._fields_ if k != "pad_"}
+
+    def kv_last_error(self) -> str:
+        return lib().kv_last_error(self._h).decode()
+
+    # -- convenience for verification (no data path): the host pool as a numpy view
+    def host_array(self) -> np.ndarray:
+        base, nbytes = self.kv_host_ptr()
+        buf = (C.c_uint8 * nbytes).from_address(base)
+        return np.frombuffer(buf, dtype=np.uint8)

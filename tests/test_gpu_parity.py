@@ -1,0 +1,272 @@
+"""GPU parity: the CUDA library, called through its C ABI, against the CPU oracle, bit for bit."""
+import itertools
+
+import numpy as np
+import pytest
+
+from paper_2601_20309_b200 import workload as W
+
+pytestmark = pytest.mark.gpu
+
+PATHS = {"zerocopy": 1, "staged": 2, "ce2d": 3, "naive": 4}
+
+
+def _pair(*a, **k):
+    from gpu_harness import Pair
+    return Pair(*a, **k)
+
+
+@pytest.mark.parametrize("path", list(PATHS))
+@pytest.mark.parametrize("flags", [0, 2, 4, 6], ids=["bulk", "ldst", "bulk-fused", "ldst-fused"])
+@pytest.mark.parametrize("layout", [0, 1], ids=["hostblockfirst", "hostlayerfirst"])
+def test_config1_tiny_rotation(path, flags, layout):
+    if path != "zerocopy" and flags & 4:
+        pytest.skip("fused launch exists on the zero-copy path only")
+    if path in ("ce2d", "naive") and flags:
+        pytest.skip("no kernel on this path")
+    w = W.config1_tiny()
+    p = _pair(w.shape, w.nb_gpu, w.nb_host, seed=w.seed, host_layout=layout, path=PATHS[path], flags=flags)
+    try:
+        assert p.rotate_both(w.steps[0]) == 0
+        p.assert_equal(f"tiny rotate {path}")
+        st = p.pool.kv_get_stats()
+        assert st["bytes_out"] == w.steps[0].n_out * w.shape.block_bytes
+        assert st["bytes_in"] == w.steps[0].n_in * w.shape.block_bytes
+        assert st["device_status"] == 0
+        if path in ("zerocopy", "staged"):
+            assert st["kernel_launches"] >= 1
+        # single directions
+        r = w.steps[0]
+        free_h = np.setdiff1d(np.arange(w.nb_host), np.concatenate([r.out_host, r.in_host]))[:10].astype(np.int32)
+        src_g = r.in_gpu[:10]
+        assert p.oracle.swap_out(src_g, free_h) == 0
+        assert p.pool.kv_swap_out(src_g, free_h) == 0
+        p.assert_equal("single swap-out")
+        dst_g = r.out_gpu[:10]
+        assert p.oracle.swap_in(free_h, dst_g) == 0
+        assert p.pool.kv_swap_in(free_h, dst_g) == 0
+        p.assert_equal("single swap-in")
+    finally:
+        p.close()
+
+
+@pytest.mark.parametrize("dims", [(3, 5, 3, 72), (1, 20, 8, 128), (2, 24, 8, 128), (5, 1, 1, 8), (2, 64, 8, 128)],
+                         ids=lambda d: "L%d_bs%d_H%d_D%d" % d)
+@pytest.mark.parametrize("flags", [0, 2], ids=["bulk", "ldst"])
+@pytest.mark.parametrize("path", ["zerocopy", "staged"])
+def test_ragged_segment_sizes(dims, flags, path):
+    """Segments that are not a whole number of kernel chunks, a 16-byte segment, and a 128 KiB one."""
+    L, bs, H, D = dims
+    shape = W.KVShape(L, bs, H, D)
+    rng = np.random.default_rng(3)
+    nbg, nbh = 37, 53
+    p = _pair(shape, nbg, nbh, seed=9, path=PATHS[path], flags=flags, staging_bytes=5 * shape.block_bytes)
+    try:
+        og = rng.choice(nbg, 17, replace=False).astype(np.int32)
+        oh = rng.choice(nbh, 17, replace=False).astype(np.int32)
+        ig = np.setdiff1d(np.arange(nbg), og)[:13].astype(np.int32)
+        ih = np.setdiff1d(np.arange(nbh), oh)[:13].astype(np.int32)
+        r = W.Rotation(og, oh, ih, ig, np.zeros(1), np.zeros(1))
+        assert p.rotate_both(r) == 0
+        p.assert_equal("ragged")
+    finally:
+        p.close()
+
+
+@pytest.mark.parametrize("path", ["zerocopy", "staged", "ce2d"])
+def test_config2_scaled_8b(path):
+    """8B shape (2 MiB blocks), pools shrunk to 320/448 blocks, request lengths scaled down; the
+    paired rotation, the single swaps and the one-pair-at-a-time rotations, compared whole-pool."""
+    w = W.config2_8b(nb_gpu=320, nb_host=448, n_req=16, median=96, max_tokens=512, n_rot=4)
+    p = _pair(w.shape, w.nb_gpu, w.nb_host, seed=w.seed, path=PATHS[path])
+    try:
+        for k in ("median", "longest"):
+            g, h = w.extra["single_out"][k]
+            assert p.oracle.swap_out(g, h) == 0 and p.pool.kv_swap_out(g, h) == 0
+            h2, g2 = w.extra["single_in"][k]
+            assert p.oracle.swap_in(h2, g2) == 0 and p.pool.kv_swap_in(h2, g2) == 0
+        p.assert_equal("single swaps")
+        assert p.rotate_both(w.steps[0]) == 0
+        p.assert_equal("rotate 4+4 requests")
+        for r in w.extra["pairs"]:
+            assert p.rotate_both(r) == 0          # no sync in between: calls queue up
+        p.assert_equal("pairwise rotations")
+    finally:
+        p.close()
+
+
+@pytest.mark.parametrize("flags", [0, 4], ids=["two-streams", "fused"])
+def test_config3_scaled_70b_steps(flags):
+    """70B shape (5 MiB blocks, 160 planes), fragmented pool, 12 steps of 2 requests each way,
+    issued back to back; what step k swaps in is what step k-2 swapped out."""
+    w = W.config3_70b(nb_gpu=160, nb_host=240, n_req=8, median=96, max_tokens=256, n_steps=12, per_step=2)
+    p = _pair(w.shape, w.nb_gpu, w.nb_host, seed=w.seed, path=1, flags=flags)
+    try:
+        for k, r in enumerate(w.steps):
+            assert p.rotate_both(r) == 0
+            if k % 5 == 4:
+                p.assert_equal(f"step {k}")
+        p.assert_equal("final")
+    finally:
+        p.close()
+
+
+@pytest.mark.parametrize("bs", [8, 16, 32, 64])
+@pytest.mark.parametrize("contig", [True, False], ids=["contiguous", "permuted"])
+def test_config4_sweep_cells_small(bs, contig):
+    w = W.config4_sweep_case(bs, contig, 48e6, num_layers=8)
+    for path in ("zerocopy", "staged", "ce2d"):
+        p = _pair(w.shape, w.nb_gpu, w.nb_host, seed=w.seed, path=PATHS[path], staging_bytes=16 << 20)
+        try:
+            assert p.rotate_both(w.steps[0]) == 0
+            p.assert_equal(f"sweep bs{bs} {path}")
+        finally:
+            p.close()
+
+
+def test_config5_replay_scaled():
+    """Replay lists (swap-outs, swap-ins, growth, empty steps) on a shrunk shape, queued without
+    syncing.  Blocks a request grows into keep whatever bytes the pool held there: whole blocks
+    move, filled or not, so the comparison stays bit-exact."""
+    w = W.config5_replay(rate=2.0, n_steps=400, shape=W.KVShape(2, 16, 2, 64), duration_s=25.0, max_tokens=1024)
+    assert sum(1 for s in w.steps if s.n_out and s.n_in) > 3
+    p = _pair(w.shape, w.nb_gpu, w.nb_host, seed=w.seed, path=1)
+    try:
+        for k, r in enumerate(w.steps):
+            assert p.rotate_both(r) == 0
+            if k % 100 == 99:
+                p.assert_equal(f"replay step {k}")
+        p.assert_equal("replay final")
+    finally:
+        p.close()
+
+
+def test_back_to_back_calls_with_cross_direction_dependencies():
+    """swap_out(g->h) immediately followed by swap_in(h->g2) with no sync: the library must order the
+    second after the first (the host block is written, then read).  Then the reverse dependency."""
+    shape = W.KVShape(4, 16, 8, 128)
+    p = _pair(shape, 64, 64, seed=5, path=1)
+    rng = np.random.default_rng(0)
+    try:
+        for _ in range(6):
+            g = rng.choice(64, 12, replace=False).astype(np.int32)
+            h = rng.choice(64, 12, replace=False).astype(np.int32)
+            g2 = rng.choice(64, 12, replace=False).astype(np.int32)
+            assert p.oracle.swap_out(g, h) == 0 and p.pool.kv_swap_out(g, h) == 0
+            assert p.oracle.swap_in(h, g2) == 0 and p.pool.kv_swap_in(h, g2) == 0       # RAW on host blocks
+            h3 = rng.choice(64, 12, replace=False).astype(np.int32)
+            assert p.oracle.swap_out(g2, h3) == 0 and p.pool.kv_swap_out(g2, h3) == 0   # RAW on device blocks
+        p.assert_equal("dependent call chain")
+    finally:
+        p.close()
+
+
+@pytest.mark.parametrize("path", ["zerocopy", "ce2d"])
+def test_overlapping_rotate_needs_flag_and_matches_sequential_semantics(path):
+    shape = W.KVShape(2, 16, 8, 128)
+    rng = np.random.default_rng(2)
+    og = np.array([3, 7, 11, 15, 19], np.int32)
+    oh = np.array([1, 2, 3, 4, 5], np.int32)
+    ih = np.array([20, 2, 21, 4, 22, 23], np.int32)         # 2 and 4 are written by the swap-out
+    ig = np.array([7, 30, 31, 15, 32, 33], np.int32)        # 7 and 15 are swap-out sources
+    r = W.Rotation(og, oh, ih, ig, np.zeros(1), np.zeros(1))
+    p = _pair(shape, 40, 40, seed=6, path=PATHS[path])
+    try:
+        before_g, before_h = p.gpu_bytes().copy(), p.pool.host_array().copy()
+        assert p.rotate_both(r) == -4
+        p.pool.kv_sync()
+        assert np.array_equal(p.gpu_bytes(), before_g) and np.array_equal(p.pool.host_array(), before_h)
+    finally:
+        p.close()
+    p = _pair(shape, 40, 40, seed=6, path=PATHS[path], flags=1)
+    try:
+        assert p.rotate_both(r, allow_overlap=True) == 0
+        p.assert_equal("overlapping rotate")
+    finally:
+        p.close()
+
+
+def test_validation_errors_move_nothing():
+    shape = W.KVShape(2, 16, 8, 128)
+    p = _pair(shape, 16, 24, seed=7, path=1)
+    try:
+        g0, h0 = p.gpu_bytes().copy(), p.pool.host_array().copy()
+        P = p.pool
+        assert P.kv_swap_out([0, 16], [0, 1], check=False) == -2
+        assert P.kv_swap_out([0, 1], [0, 24], check=False) == -2
+        assert P.kv_swap_out([0, -1], [0, 1], check=False) == -2
+        assert P.kv_swap_out([0, 1], [5, 5], check=False) == -3
+        assert P.kv_swap_in([0, 1], [5, 5], check=False) == -3
+        assert P.kv_rotate([0], [1], [2], [0], check=False) == -4
+        assert P.kv_rotate([0], [1], [1], [2], check=False) == -4
+        assert "race" in P.kv_last_error()
+        assert P.kv_swap_out([1, 1], [2, 3], check=False) == 0       # duplicate sources are fine
+        assert p.oracle.swap_out([1, 1], [2, 3]) == 0
+        assert P.kv_rotate([], [], [], [], check=False) == 0
+        assert P.kv_swap_out([], [], check=False) == 0 and P.kv_swap_in([], [], check=False) == 0
+        p.assert_equal("after refused calls")
+        assert not np.array_equal(p.pool.host_array(), h0)           # the valid call did move bytes
+        assert np.array_equal(p.gpu_bytes(), g0)
+    finally:
+        p.close()
+
+
+def test_whole_pool_in_one_call_and_device_leg():
+    """n = every block of the device pool; then gather/scatter through a contiguous device buffer."""
+    import torch
+    shape = W.KVShape(3, 16, 8, 128)
+    nbg, nbh = 48, 48
+    p = _pair(shape, nbg, nbh, seed=8, path=1)
+    try:
+        rng = np.random.default_rng(1)
+        g = rng.permutation(nbg).astype(np.int32)
+        h = rng.permutation(nbh).astype(np.int32)
+        assert p.oracle.swap_out(g, h) == 0 and p.pool.kv_swap_out(g, h) == 0
+        p.assert_equal("whole pool out")
+        g2 = rng.permutation(nbg).astype(np.int32)
+        assert p.oracle.swap_in(h, g2) == 0 and p.pool.kv_swap_in(h, g2) == 0
+        p.assert_equal("whole pool in")
+        # device leg: gather listed blocks into a contiguous block-first buffer
+        ids = rng.choice(nbg, 20, replace=False).astype(np.int32)
+        buf = torch.zeros(20 * shape.block_bytes, dtype=torch.uint8, device="cuda:0")
+        assert p.pool.kv_gather_blocks(ids, buf.data_ptr()) == 0
+        p.pool.kv_sync()
+        got = buf.cpu().numpy().reshape(20, shape.block_bytes)
+        for k, b in enumerate(ids):
+            assert np.array_equal(got[k], p.oracle.g_block(int(b)))
+        # scatter them back to other ids: equals a swap-in from a block-first host model
+        dst = rng.permutation(nbg)[:20].astype(np.int32)
+        expect = {int(d): p.oracle.g_block(int(s)).copy() for s, d in zip(ids, dst)}
+        assert p.pool.kv_scatter_blocks(buf.data_ptr(), dst) == 0
+        p.pool.kv_sync()
+        gb = p.gpu_bytes()
+        seg = p.oracle.seg
+        for d, want in expect.items():
+            have = np.concatenate([gb[p.oracle.dev_off(l, kv, d):p.oracle.dev_off(l, kv, d) + seg]
+                                   for l in range(shape.num_layers) for kv in range(2)])
+            assert np.array_equal(have, want)
+        touched = set(int(x) for x in dst)
+        for b in range(nbg):
+            if b not in touched:
+                o = p.oracle.dev_off(1, 1, b)
+                assert np.array_equal(gb[o:o + seg], p.oracle.G[o:o + seg])
+    finally:
+        p.close()
+
+
+def test_gpu_fill_twin_matches_cpu_generator():
+    """The GPU pool-fill helper must write exactly what workload.block_words generates."""
+    import torch
+    from paper_2601_20309_b200 import poolfill as F
+    shape = W.KVShape(3, 8, 2, 64)
+    nb = 11
+    dev = torch.zeros(nb * shape.block_bytes, dtype=torch.uint8, device="cuda:0")
+    lay = F.Layout.device(dev.data_ptr(), shape, nb)
+    F.fill_blocks(lay, 77, W.POOL_GPU, nb)
+    got = dev.cpu().numpy().view(np.uint16).reshape(2 * shape.num_layers, nb, shape.words_per_plane)
+    for b in range(nb):
+        want = W.block_words(77, W.POOL_GPU, b, shape.words_per_block).reshape(2 * shape.num_layers, -1)
+        assert np.array_equal(got[:, b, :], want)
+    sums = F.checksum_blocks(lay, nb)
+    for b in range(nb):
+        assert sums[b] == F.checksum_words(W.block_words(77, W.POOL_GPU, b, shape.words_per_block))
