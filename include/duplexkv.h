@@ -81,11 +81,14 @@ typedef struct {
     int32_t device_id;
     void   *stream_out;     /* cudaStream_t or NULL (library creates a non-blocking stream)               */
     void   *stream_in;      /* likewise; must differ from stream_out for the directions to overlap        */
-    int32_t path;           /* KV_PATH_*                                                                  */
+    int32_t path;           /* KV_PATH_* of the swap-out direction, and of swap-in unless path_in is set  */
     int32_t flags;          /* KV_FLAG_*                                                                  */
     int32_t ctas_out;       /* CTAs of the swap-out kernel, 0 = default for the path                      */
     int32_t ctas_in;        /* CTAs of the swap-in kernel, 0 = default                                    */
     int64_t staging_bytes;  /* per-direction HBM staging buffer of the STAGED path, 0 = 64 MiB            */
+    int32_t path_in;        /* KV_PATH_* of the swap-in direction; KV_PATH_AUTO (0) = same as `path`      */
+    int32_t ce_streams;     /* streams per direction that the copy-engine paths spread their transfers
+                               over (1..4), 0 = 1                                                         */
 } kv_pool_config_t;
 
 typedef struct {

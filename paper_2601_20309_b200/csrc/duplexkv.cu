@@ -19,6 +19,7 @@
 namespace {
 
 constexpr int KV_SLOTS = 8;            // descriptor / event ring depth per direction
+constexpr int KV_MAX_CE_STREAMS = 4;
 constexpr int BULK_STAGE = 16384;      // bytes per shared-memory stage of the bulk kernel
 constexpr int BULK_NS = 8;             // stages
 constexpr int BULK_AHEAD = 5;          // loads in flight ahead of the stores
@@ -39,7 +40,13 @@ struct DirState {
     uint64_t done = 0;                 // latest call known to be complete
     uint8_t *stage = nullptr;          // HBM staging (STAGED path), allocated on first use
     int ctas = 0;
-    int last_path = 0;
+    int path = 0;                      // configured path of this direction (may be KV_PATH_AUTO)
+    // copy-engine paths spread their transfers over nsub streams: sub[0] is `stream`, the others
+    // are forked from it and joined back with events, so per-transfer start-up gaps overlap
+    int nsub = 1;
+    cudaStream_t sub[KV_MAX_CE_STREAMS] = {};
+    cudaEvent_t fork_ev = nullptr;
+    cudaEvent_t join_ev[KV_MAX_CE_STREAMS] = {};
 };
 
 }  // namespace
@@ -227,13 +234,34 @@ struct DirCall {
     // copy-engine issue state (CE paths are issued in slices so the two directions interleave)
     int64_t ce_next = 0;
     int64_t chunk_lo = 0;
+    bool chunk_open = false;
+    unsigned rr = 0;                   // round-robin cursor over the direction's CE streams
 };
 
-int resolve_path(const kv_pool *p)
+int resolve_path(const kv_pool *p, int d)
 {
-    int path = p->cfg.path;
+    int path = p->dir[d].path;
     if (path == KV_PATH_AUTO) path = kv_path_for(p->seg);
     return path;
+}
+
+// fork: the extra streams of a CE direction wait for everything issued so far on its main stream
+int32_t ce_fork(kv_pool *p, DirState &s)
+{
+    if (s.nsub <= 1) return KV_OK;
+    KV_CUDA(p, cudaEventRecord(s.fork_ev, s.stream));
+    for (int k = 1; k < s.nsub; ++k) KV_CUDA(p, cudaStreamWaitEvent(s.sub[k], s.fork_ev, 0));
+    return KV_OK;
+}
+
+// join: the main stream waits for everything issued on the extra streams
+int32_t ce_join(kv_pool *p, DirState &s)
+{
+    for (int k = 1; k < s.nsub; ++k) {
+        KV_CUDA(p, cudaEventRecord(s.join_ev[k], s.sub[k]));
+        KV_CUDA(p, cudaStreamWaitEvent(s.stream, s.join_ev[k], 0));
+    }
+    return KV_OK;
 }
 
 int32_t begin_dir(kv_pool *p, DirCall &c, bool wait_other)
@@ -268,8 +296,11 @@ int32_t begin_dir(kv_pool *p, DirCall &c, bool wait_other)
             }
         }
     }
+    if (c.path == KV_PATH_CE2D || c.path == KV_PATH_NAIVE) {
+        int32_t rc = ce_fork(p, s);
+        if (rc != KV_OK) return rc;
+    }
     s.issued = seq;
-    s.last_path = c.path;
     note_use(p, c.d, c.gpu_ids, c.host_ids, c.n, seq);
     return KV_OK;
 }
@@ -277,6 +308,10 @@ int32_t begin_dir(kv_pool *p, DirCall &c, bool wait_other)
 int32_t end_dir(kv_pool *p, DirCall &c)
 {
     DirState &s = p->dir[c.d];
+    if (c.path == KV_PATH_CE2D || c.path == KV_PATH_NAIVE) {
+        int32_t rc = ce_join(p, s);
+        if (rc != KV_OK) return rc;
+    }
     KV_CUDA(p, cudaEventRecord(s.ev_end[c.slot], s.stream));
     const int64_t bytes = c.n * p->blk;
     if (c.d == 0) {
@@ -326,7 +361,7 @@ int32_t ce_issue_some(kv_pool *p, DirCall &c, int budget, bool &finished)
             const int64_t i = c.ce_next / p->planes, pl = c.ce_next % p->planes;
             uint8_t *dv = p->dev + (pl * p->cfg.num_gpu_blocks + c.gpu_ids[i]) * p->seg;
             uint8_t *hv = host_block_ptr(p, c.host_ids[i]) + pl * (int64_t)host_pitch(p);
-            KV_CUDA(p, cudaMemcpyAsync(c.d == 0 ? hv : dv, c.d == 0 ? dv : hv, (size_t)p->seg, kind, s.stream));
+            KV_CUDA(p, cudaMemcpyAsync(c.d == 0 ? hv : dv, c.d == 0 ? dv : hv, (size_t)p->seg, kind, s.sub[i % s.nsub]));
             p->stats.ce_copies++;
             c.ce_next++;
         }
@@ -340,10 +375,11 @@ int32_t ce_issue_some(kv_pool *p, DirCall &c, int budget, bool &finished)
             uint8_t *dv = p->dev + (int64_t)c.gpu_ids[i] * p->seg;
             uint8_t *hv = host_block_ptr(p, c.host_ids[i]);
             const size_t dpitch = (size_t)(p->cfg.num_gpu_blocks * p->seg);
+            cudaStream_t cs = s.sub[i % s.nsub];
             if (c.d == 0)
-                KV_CUDA(p, cudaMemcpy2DAsync(hv, host_pitch(p), dv, dpitch, (size_t)p->seg, (size_t)p->planes, kind, s.stream));
+                KV_CUDA(p, cudaMemcpy2DAsync(hv, host_pitch(p), dv, dpitch, (size_t)p->seg, (size_t)p->planes, kind, cs));
             else
-                KV_CUDA(p, cudaMemcpy2DAsync(dv, dpitch, hv, host_pitch(p), (size_t)p->seg, (size_t)p->planes, kind, s.stream));
+                KV_CUDA(p, cudaMemcpy2DAsync(dv, dpitch, hv, host_pitch(p), (size_t)p->seg, (size_t)p->planes, kind, cs));
             p->stats.ce_copies++;
             c.ce_next++;
         }
@@ -367,30 +403,40 @@ int32_t ce_issue_some(kv_pool *p, DirCall &c, int budget, bool &finished)
         kd.pairs = c.aux_dev + lo;
         kd.n = (int)(hi - lo);
         kd.ctas = clamp_ctas(job, kd, p->sm_count);
-        if (c.d == 0 && c.ce_next == lo) KV_CUDA(p, launch_job(p, job, s.stream));
-        if (c.ce_next < lo) c.ce_next = lo;
+        if (c.ce_next == lo && !c.chunk_open) {
+            // out: gather into the staging buffer first; both: the extra streams start after what
+            // the main stream has done so far (the gather, or the previous chunk's scatter)
+            if (c.d == 0) KV_CUDA(p, launch_job(p, job, s.stream));
+            int32_t rc = ce_fork(p, s);
+            if (rc != KV_OK) return rc;
+            c.chunk_open = true;
+        }
         while (budget > 0 && c.ce_next < hi) {
             int64_t k = c.ce_next, run = 1;
             if (p->cfg.host_layout == KV_HOST_BLOCK_FIRST) {
                 while (k + run < hi && c.host_ids[k + run] == c.host_ids[k] + run) ++run;
                 uint8_t *hv = host_block_ptr(p, c.host_ids[k]);
                 uint8_t *sv = s.stage + (k - lo) * p->blk;
-                KV_CUDA(p, cudaMemcpyAsync(c.d == 0 ? hv : sv, c.d == 0 ? sv : hv, (size_t)(run * p->blk), kind, s.stream));
+                KV_CUDA(p, cudaMemcpyAsync(c.d == 0 ? hv : sv, c.d == 0 ? sv : hv, (size_t)(run * p->blk), kind, s.sub[c.rr++ % s.nsub]));
             } else {
                 uint8_t *hv = host_block_ptr(p, c.host_ids[k]);
                 uint8_t *sv = s.stage + (k - lo) * p->blk;
+                cudaStream_t cs = s.sub[c.rr++ % s.nsub];
                 if (c.d == 0)
-                    KV_CUDA(p, cudaMemcpy2DAsync(hv, host_pitch(p), sv, (size_t)p->seg, (size_t)p->seg, (size_t)p->planes, kind, s.stream));
+                    KV_CUDA(p, cudaMemcpy2DAsync(hv, host_pitch(p), sv, (size_t)p->seg, (size_t)p->seg, (size_t)p->planes, kind, cs));
                 else
-                    KV_CUDA(p, cudaMemcpy2DAsync(sv, (size_t)p->seg, hv, host_pitch(p), (size_t)p->seg, (size_t)p->planes, kind, s.stream));
+                    KV_CUDA(p, cudaMemcpy2DAsync(sv, (size_t)p->seg, hv, host_pitch(p), (size_t)p->seg, (size_t)p->planes, kind, cs));
             }
             p->stats.ce_copies++;
             c.ce_next += run;
             --budget;
         }
         if (c.ce_next >= hi) {
+            int32_t rc = ce_join(p, s);
+            if (rc != KV_OK) return rc;
             if (c.d == 1) KV_CUDA(p, launch_job(p, job, s.stream));
             c.chunk_lo = hi;
+            c.chunk_open = false;
         }
     }
     finished = c.chunk_lo >= c.n;
@@ -438,7 +484,7 @@ int32_t run_calls(kv_pool *p, DirCall *calls, int ncalls, const bool *wait_other
 {
     p->union_slot[0] = p->union_slot[1] = -1;
     for (int k = 0; k < ncalls; ++k) {
-        calls[k].path = resolve_path(p);
+        calls[k].path = resolve_path(p, calls[k].d);
         if (fused && calls[k].d == 1) {
             // the fused launch runs on the out stream: order it after earlier swap-ins, and later swap-ins after it
             DirState &in = p->dir[1];
@@ -518,9 +564,11 @@ int32_t kv_pool_create(const kv_pool_config_t *cfg, kv_pool_t **out)
         return fail(nullptr, KV_ERR_INVALID_ARG, "host_base must be 4096-byte aligned");
     if (cfg->host_layout != KV_HOST_BLOCK_FIRST && cfg->host_layout != KV_HOST_LAYER_FIRST)
         return fail(nullptr, KV_ERR_INVALID_ARG, "unknown host_layout");
-    if (cfg->path < KV_PATH_AUTO || cfg->path > KV_PATH_NAIVE) return fail(nullptr, KV_ERR_INVALID_ARG, "unknown path");
-    if (cfg->ctas_out < 0 || cfg->ctas_in < 0 || cfg->staging_bytes < 0)
-        return fail(nullptr, KV_ERR_INVALID_ARG, "negative tuning value");
+    if (cfg->path < KV_PATH_AUTO || cfg->path > KV_PATH_NAIVE || cfg->path_in < KV_PATH_AUTO || cfg->path_in > KV_PATH_NAIVE)
+        return fail(nullptr, KV_ERR_INVALID_ARG, "unknown path");
+    if (cfg->ctas_out < 0 || cfg->ctas_in < 0 || cfg->staging_bytes < 0 || cfg->ce_streams < 0 ||
+        cfg->ce_streams > KV_MAX_CE_STREAMS)
+        return fail(nullptr, KV_ERR_INVALID_ARG, "tuning value out of range");
 
     KV_CUDA(nullptr, cudaSetDevice(cfg->device_id));
     kv_pool *p = new (std::nothrow) kv_pool();
@@ -595,6 +643,14 @@ int32_t kv_pool_create(const kv_pool_config_t *cfg, kv_pool_t **out)
             KV_CREATE_CUDA(cudaEventCreate(&s.ev_end[k]));
         }
         s.ctas = want_ctas[d] > 0 ? want_ctas[d] : 32;
+        s.path = (d == 1 && cfg->path_in != KV_PATH_AUTO) ? cfg->path_in : cfg->path;
+        s.nsub = cfg->ce_streams > 0 ? cfg->ce_streams : 1;
+        s.sub[0] = s.stream;
+        KV_CREATE_CUDA(cudaEventCreateWithFlags(&s.fork_ev, cudaEventDisableTiming));
+        for (int k = 1; k < s.nsub; ++k) {
+            KV_CREATE_CUDA(cudaStreamCreateWithFlags(&s.sub[k], cudaStreamNonBlocking));
+            KV_CREATE_CUDA(cudaEventCreateWithFlags(&s.join_ev[k], cudaEventDisableTiming));
+        }
     }
     KV_CREATE_CUDA(cudaFuncSetAttribute(kv_copy_bulk<BULK_STAGE, BULK_NS, BULK_AHEAD>,
                                         cudaFuncAttributeMaxDynamicSharedMemorySize, BULK_STAGE * BULK_NS));
@@ -628,6 +684,12 @@ int32_t kv_pool_destroy(kv_pool_t *p)
             if (s.ev_start[k]) (void)cudaEventDestroy(s.ev_start[k]);
             if (s.ev_end[k]) (void)cudaEventDestroy(s.ev_end[k]);
         }
+        for (int k = 1; k < KV_MAX_CE_STREAMS; ++k) {
+            if (s.sub[k]) (void)cudaStreamSynchronize(s.sub[k]);
+            if (s.sub[k]) (void)cudaStreamDestroy(s.sub[k]);
+            if (s.join_ev[k]) (void)cudaEventDestroy(s.join_ev[k]);
+        }
+        if (s.fork_ev) (void)cudaEventDestroy(s.fork_ev);
         if (s.ring_host) (void)cudaFreeHost(s.ring_host);
         if (s.ring_dev) (void)cudaFree(s.ring_dev);
         if (s.stage) (void)cudaFree(s.stage);
@@ -708,7 +770,8 @@ int32_t kv_rotate(kv_pool_t *p, const int32_t *out_gpu, const int32_t *out_host,
         calls[1].n = n_in;
         const bool wait[2] = {conflicts_with_other(p, 0, out_gpu, out_host, n_out),
                               conflicts_with_other(p, 1, in_gpu, in_host, n_in)};
-        const bool fused = (p->cfg.flags & KV_FLAG_FUSED_ROTATE) && resolve_path(p) == KV_PATH_ZEROCOPY && !wait[0] && !wait[1];
+        const bool fused = (p->cfg.flags & KV_FLAG_FUSED_ROTATE) && resolve_path(p, 0) == KV_PATH_ZEROCOPY &&
+                           resolve_path(p, 1) == KV_PATH_ZEROCOPY && !wait[0] && !wait[1];
         return run_calls(p, calls, 2, wait, fused);
     }
     // overlap allowed: the conflict-free swap-ins run beside the swap-out, the others after it
