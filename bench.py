@@ -37,6 +37,9 @@ from paper_2601_20309_b200 import workload as W         # noqa: E402
 
 METRIC = "full-duplex KV swap GB/s (out+in)"
 UNIT = "GB/s"
+# dram__bytes_read.sum + dram__bytes_write.sum of one pack launch, scaled from the ncu capture on the
+# small case (traffic grows with the bytes moved); None until counters exist for the current kernel
+NCU_TRAFFIC_PER_LAUNCH = None
 
 
 # ------------------------------------------------------------------------------------------------ helpers
@@ -187,21 +190,14 @@ def run_ours(args, rank: int, local_rank: int, world: int) -> None:
             dist.barrier()
         torch.cuda.synchronize()
 
-    def max_over_ranks(x: float) -> float:
+    def reduce(x: float, op: str) -> float:
         if dist is None:
             return x
         t = torch.tensor([x], dtype=torch.float64, device=dev)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX if op == "max" else dist.ReduceOp.SUM)
         return float(t.item())
 
-    def sum_over_ranks(x: float) -> float:
-        if dist is None:
-            return x
-        t = torch.tensor([x], dtype=torch.float64, device=dev)
-        dist.all_reduce(t, op=dist.ReduceOp.SUM)
-        return float(t.item())
-
-    # ---- roofline denominators, measured here
+    # ---- host-link denominators, measured in this process (again after the timed region)
     probe = B.kv_probe_link(local_rank, 256 << 20, 4)
     peaks = measured_peaks()
 
@@ -226,14 +222,15 @@ def run_ours(args, rank: int, local_rank: int, world: int) -> None:
     device_pool = torch.empty(nb_gpu * shape.block_bytes, dtype=torch.uint8, device=dev)
     t0 = time.perf_counter()
     pool = B.KVPool(shape.num_layers, shape.block_size, shape.kv_heads, shape.head_dim, nb_gpu, nb_host,
-                    device_pool.data_ptr(), device_id=local_rank, path=args.path, flags=args.flags,
-                    ctas_out=args.ctas, ctas_in=args.ctas)
+                    device_pool.data_ptr(), device_id=local_rank, path=args.path,
+                    flags=args.flags | B.KV_FLAG_TIME_KERNELS, ctas_out=args.ctas, ctas_in=args.ctas,
+                    staging_bytes=args.staging_mib << 20)
     pin_s = time.perf_counter() - t0
     host_base, host_bytes = pool.kv_host_ptr()
-    # seeded content in both pools (GPU twin of the CPU generator; verified against it in the tests)
+    # seeded content in both pools (GPU twin of the CPU generator; verified against it in the tests);
+    # mapped pinned memory has the same address on the device (unified addressing)
     F.fill_blocks(F.Layout.device(device_pool.data_ptr(), shape, nb_gpu), w.seed, W.POOL_GPU, nb_gpu, device=dev)
-    host_dev_ptr = host_base       # unified addressing: mapped pinned memory has the same address on the device
-    F.fill_blocks(F.Layout.host(host_dev_ptr, shape, nb_host), w.seed, W.POOL_HOST, nb_host, device=dev)
+    F.fill_blocks(F.Layout.host(host_base, shape, nb_host), w.seed, W.POOL_HOST, nb_host, device=dev)
 
     og, oh, ih, ig = (np.ascontiguousarray(x, np.int32) for x in (rot.out_gpu, rot.out_host, rot.in_host, rot.in_gpu))
     args_raw = (ptr(og), ptr(oh), len(og), ptr(ih), ptr(ig), len(ig))
@@ -246,7 +243,7 @@ def run_ours(args, rank: int, local_rank: int, world: int) -> None:
 
     for _ in range(args.warmup):
         step()
-    launches0 = pool.kv_get_stats()["kernel_launches"]
+    st0 = pool.kv_get_stats()
     sampler = ClockSampler(local_rank)
     sampler.start()
     barrier()
@@ -259,37 +256,60 @@ def run_ours(args, rank: int, local_rank: int, world: int) -> None:
     wall_s = time.perf_counter() - t0
     clocks = sampler.stop()
     st = pool.kv_get_stats()
-    launches = st["kernel_launches"] - launches0
+    launches = st["kernel_launches"] - st0["kernel_launches"]
+    ce_copies = st["ce_copies"] - st0["ce_copies"]
+    k_ms = st["timed_kernel_ms"] - st0["timed_kernel_ms"]
+    k_bytes = st["timed_kernel_bytes"] - st0["timed_kernel_bytes"]
+    k_n = st["timed_kernels"] - st0["timed_kernels"]
 
-    dev_total_ms = max_over_ranks(float(np.sum(dev_ms)))
-    wall_total_s = max_over_ranks(wall_s)
-    job_bytes = sum_over_ranks(float(bytes_out + bytes_in)) * args.steps
+    dev_total_ms = reduce(float(np.sum(dev_ms)), "max")
+    wall_total_s = reduce(wall_s, "max")
+    job_bytes = reduce(float(bytes_out + bytes_in), "sum") * args.steps
     value = M.gbs(job_bytes, dev_total_ms)
     e2e_value = job_bytes / wall_total_s / 1e9
 
     extra = {}
     if rank == 0:
-        # ---- each direction alone (Table 1's "u" rows): the same lists, one direction per call
-        uni = {}
-        for name, fn, nb in (("out", lambda: pool.kv_swap_out(og, oh), bytes_out),
-                             ("in", lambda: pool.kv_swap_in(ih, ig), bytes_in)):
+        def timed(fn, reps=3):
             ts = []
-            for _ in range(3):
+            for _ in range(reps):
                 fn()
                 pool.kv_sync()
                 ts.append(pool.kv_get_stats()["last_union_ms"])
-            uni[name] = M.gbs(nb, min(ts))
+            return min(ts)
+
+        probe2 = B.kv_probe_link(local_rank, 256 << 20, 4)
+        # ---- every path on the same lists: each direction alone ("u") and both at once ("b"),
+        #      the conventions of the paper's bandwidth table
+        paths = {}
+        path_list = [("staged", B.KV_PATH_STAGED), ("zerocopy", B.KV_PATH_ZEROCOPY), ("ce2d", B.KV_PATH_CE2D)]
+        if not args.quick:
+            path_list.append(("naive", B.KV_PATH_NAIVE))
+        for name, pid in path_list:
+            pool.kv_pool_set_path(pid, pid)
+            reps = 1 if name == "naive" else 3
+            # the per-segment path is measured on the first 256 blocks of each list (16 384 transfers each way)
+            cut = 256 if name == "naive" else None
+            a = (og[:cut], oh[:cut], ih[:cut], ig[:cut])
+            bo, bi_ = len(a[0]) * shape.block_bytes, len(a[3]) * shape.block_bytes
+            t_o = timed(lambda: pool.kv_swap_out(a[0], a[1]), reps)
+            t_i = timed(lambda: pool.kv_swap_in(a[2], a[3]), reps)
+            t_b = timed(lambda: pool.kv_rotate(*a), reps)
+            paths[name] = {"out_u_gbs": M.gbs(bo, t_o), "in_u_gbs": M.gbs(bi_, t_i), "both_b_gbs": M.gbs(bo + bi_, t_b),
+                           "e2e_ms_serial_u": t_o + t_i, "e2e_ms_concurrent_b": t_b, "blocks_each_way": len(a[0])}
+        pool.kv_pool_set_path(args.path, args.path)
+        # ---- the same payload with neighbouring host ids (what a run-based host allocator would hand out)
+        oh_c = np.arange(len(og), dtype=np.int32)
+        ih_c = np.arange(nb_host - len(ig), nb_host, dtype=np.int32)
+        t_c = timed(lambda: pool.kv_rotate(og, oh_c, ih_c, ig))
+        contiguous_host = M.gbs(bytes_out + bytes_in, t_c)
+        F.fill_blocks(F.Layout.host(host_base, shape, nb_host), w.seed, W.POOL_HOST, len(og), device=dev)   # restore what it overwrote
         # ---- single swaps of the median-length and the longest request
         singles = {}
         for key, which in (("single_out", "out"), ("single_in", "in")):
             for k, (a, b) in w.extra[key].items():
-                ts = []
-                for _ in range(3):
-                    (pool.kv_swap_out(a, b) if which == "out" else pool.kv_swap_in(a, b))
-                    pool.kv_sync()
-                    ts.append(pool.kv_get_stats()["last_union_ms"])
-                singles[f"{which}_{k}"] = {"blocks": len(a), "gbs": M.gbs(len(a) * shape.block_bytes, min(ts)),
-                                           "ms": min(ts)}
+                t = timed((lambda a=a, b=b: pool.kv_swap_out(a, b)) if which == "out" else (lambda a=a, b=b: pool.kv_swap_in(a, b)))
+                singles[f"{which}_{k}"] = {"blocks": len(a), "gbs": M.gbs(len(a) * shape.block_bytes, t), "ms": t}
         # ---- per-request rotate latency: one request out + one in per call, call entry to completion
         lat_us, lat_blocks = [], []
         for r in w.extra["pairs"] * 2:
@@ -301,24 +321,22 @@ def run_ours(args, rank: int, local_rank: int, world: int) -> None:
             lat_us.append((time.perf_counter() - t1) * 1e6)
             lat_blocks.append(len(a[0]) + len(a[3]))
         lat_us = lat_us[len(lat_us) // 2:]       # second pass (first pass warms the path)
-        # ---- device-side gather/scatter (HBM <-> contiguous HBM), the kernel half of the staged path
-        ids = og
-        stage = torch.empty(len(ids) * shape.block_bytes, dtype=torch.uint8, device=dev)
+        lat_blocks = lat_blocks[len(lat_blocks) // 2:]
+        # ---- device-side gather / scatter on their own (HBM <-> contiguous HBM), whole list in one launch
+        stage = torch.empty(len(og) * shape.block_bytes, dtype=torch.uint8, device=dev)
         leg = {}
-        for name, fn in (("gather", lambda: pool.kv_gather_blocks(ids, stage.data_ptr())),
-                         ("scatter", lambda: pool.kv_scatter_blocks(stage.data_ptr(), ig[:len(ids)]))):
+        for name, fn in (("gather", lambda: pool.kv_gather_blocks(og, stage.data_ptr())),
+                         ("scatter", lambda: pool.kv_scatter_blocks(stage.data_ptr(), ig[:len(og)]))):
             ts = []
             for _ in range(8):
                 fn()
                 pool.kv_sync()
                 ts.append(pool.kv_get_stats()["last_union_ms"])
             leg[name] = float(np.mean(ts[3:]))
-        n_leg = min(len(ids), len(ig))
-        leg_bytes = 2.0 * len(ids) * shape.block_bytes          # read + write
-        hbm_ach = M.gbs(leg_bytes, leg["gather"])
+        leg_bytes = 2.0 * len(og) * shape.block_bytes          # read + write
         del stage
-        extra = {"uni": uni, "singles": singles, "lat_us": lat_us, "lat_blocks": lat_blocks[len(lat_blocks) // 2:],
-                 "leg": leg, "hbm_ach": hbm_ach, "leg_bytes": leg_bytes, "n_leg": n_leg}
+        extra = {"paths": paths, "singles": singles, "lat_us": lat_us, "lat_blocks": lat_blocks, "leg": leg,
+                 "leg_bytes": leg_bytes, "probe2": probe2, "contiguous_host": contiguous_host}
 
     pool.destroy()
     del device_pool
@@ -333,9 +351,34 @@ def run_ours(args, rank: int, local_rank: int, world: int) -> None:
         cpu_1 = M.gbs(2 * 256 * shape.block_bytes, float(np.mean(t_1)) * 1e3)
 
         step_ms = dev_total_ms / args.steps
-        p_bi = probe["bi_sum_gbs"]
-        ideal_ms = M.duplex_ideal_ms(bytes_out, bytes_in, probe["d2h_gbs"], probe["h2d_gbs"], p_bi)
-        uni = extra["uni"]
+        probe2 = extra["probe2"]
+        p_bi = max(probe["bi_sum_gbs"], probe2["bi_sum_gbs"])
+        p_d2h = max(probe["d2h_gbs"], probe2["d2h_gbs"])
+        p_h2d = max(probe["h2d_gbs"], probe2["h2d_gbs"])
+        ideal_ms = M.duplex_ideal_ms(bytes_out, bytes_in, p_d2h, p_h2d, p_bi)
+        paths = extra["paths"]
+        mine = B.PATH_NAMES[st["last_path_out"]]
+        uni = paths.get(mine, paths["staged"])
+        link = {"bound": "host_link", "achieved": value / world, "peak": p_bi, "unit": "GB/s",
+                "frac": value / world / p_bi,
+                "peak_source": "pinned copy-engine probe in this process, 256 MiB transfers, both directions at once; "
+                               "the larger of the readings taken before and after the timed region (of measured)",
+                "probe_before": probe, "probe_after": probe2, "ideal_ms_per_step": ideal_ms}
+        leg_ach = M.gbs(extra["leg_bytes"], extra["leg"]["gather"])
+        if k_n > 0:
+            k_avg_ms = k_ms / k_n
+            k_ach = M.gbs(2.0 * k_bytes, k_ms)
+            roofline = {"bound": "hbm", "achieved": k_ach, "peak": peaks["hbm_gbs"], "unit": "GB/s",
+                        "frac": k_ach / peaks["hbm_gbs"], "traffic": NCU_TRAFFIC_PER_LAUNCH,
+                        "kernel": "kv_copy_bulk (pack: scattered HBM planes -> contiguous HBM staging; unpack: the reverse)",
+                        "launches_timed": int(k_n), "avg_launch_us": k_avg_ms * 1e3,
+                        "algorithmic_bytes_per_launch": 2.0 * k_bytes / k_n,
+                        "peak_source": f"MEASURED_PEAKS.json hbm_gbs ({peaks['source']}; burst copy figure)",
+                        "frac_of_nominal_8TBs": k_ach / 8000.0,
+                        "how": "CUDA events around every pack / unpack launch on the stream it runs on, inside the timed steps"}
+        else:
+            # zero-copy path: the dominant kernel crosses the host link, which is what bounds it
+            roofline = dict(link, kernel="kv_copy_bulk (zero-copy rotate)", traffic=None)
         line = {
             "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
             "warmup": args.warmup, "ms_per_step": step_ms, "higher_is_better": True, "scaling": "weak",
@@ -347,31 +390,29 @@ def run_ours(args, rank: int, local_rank: int, world: int) -> None:
                        "blocks_out": int(rot.n_out), "blocks_in": int(rot.n_in), "block_bytes": shape.block_bytes,
                        "bytes_out_per_step": bytes_out, "bytes_in_per_step": bytes_in,
                        "path_out": B.PATH_NAMES[st["last_path_out"]], "path_in": B.PATH_NAMES[st["last_path_in"]],
+                       "block_tables": "scattered ids in both pools (seeded free-list allocator)",
                        "l2": "inputs larger than L2 (3.9 GB per direction per step)", "replicas": world,
                        "pin_seconds": round(pin_s, 1)},
             "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": bytes_in + 8 * (rot.n_out + rot.n_in),
                     "d2h_bytes_per_step": bytes_out, "ms_per_step": wall_total_s * 1e3 / args.steps},
-            "gpu_launches": int(launches),
+            "gpu_launches": int(launches), "ce_transfers": int(ce_copies),
             "clocks": clocks,
-            "roofline": {"bound": "host_link", "achieved": value / world, "peak": p_bi, "unit": "GB/s",
-                         "frac": value / world / p_bi, "traffic": None,
-                         "peak_source": "pinned copy-engine probe in this process (256 MiB x 4, both directions at once)",
-                         "kernel": "kv_copy_bulk (zero-copy rotate)", "ideal_ms_per_step": ideal_ms},
-            "roofline_hbm": {"bound": "hbm", "achieved": extra["hbm_ach"], "peak": peaks["hbm_gbs"], "unit": "GB/s",
-                             "frac": extra["hbm_ach"] / peaks["hbm_gbs"], "traffic": None,
-                             "peak_source": f"MEASURED_PEAKS.json ({peaks['source']})",
-                             "frac_of_nominal_8TBs": extra["hbm_ach"] / 8000.0,
-                             "kernel": "kv_copy_bulk (device-side gather, HBM to contiguous HBM)",
-                             "gather_ms": extra["leg"]["gather"], "scatter_ms": extra["leg"]["scatter"],
-                             "algorithmic_bytes": extra["leg_bytes"]},
-            "link_probe": probe,
+            "roofline": roofline,
+            "roofline_link": link,
+            "roofline_hbm_standalone": {"bound": "hbm", "achieved": leg_ach, "peak": peaks["hbm_gbs"], "unit": "GB/s",
+                                        "frac": leg_ach / peaks["hbm_gbs"], "frac_of_nominal_8TBs": leg_ach / 8000.0,
+                                        "kernel": "kv_copy_bulk via kv_gather_blocks / kv_scatter_blocks, the whole "
+                                                  "out list in one launch",
+                                        "gather_ms": extra["leg"]["gather"], "scatter_ms": extra["leg"]["scatter"],
+                                        "algorithmic_bytes": extra["leg_bytes"]},
             "directions": {"rotate_out_gbs": M.gbs(bytes_out * args.steps, dev_total_ms),
                            "rotate_in_gbs": M.gbs(bytes_in * args.steps, dev_total_ms),
-                           "out_alone_gbs": uni["out"], "in_alone_gbs": uni["in"],
-                           "out_alone_frac_of_d2h": uni["out"] / probe["d2h_gbs"],
-                           "in_alone_frac_of_h2d": uni["in"] / probe["h2d_gbs"],
-                           "e2e_ms_serial_u": M.e2e_ms(bytes_out, bytes_in, uni["out"], uni["in"], False),
-                           "e2e_ms_concurrent_b": step_ms},
+                           "out_alone_gbs": uni["out_u_gbs"], "in_alone_gbs": uni["in_u_gbs"],
+                           "out_alone_frac_of_d2h": uni["out_u_gbs"] / p_d2h,
+                           "in_alone_frac_of_h2d": uni["in_u_gbs"] / p_h2d,
+                           "e2e_ms_serial_u": uni["e2e_ms_serial_u"], "e2e_ms_concurrent_b": step_ms},
+            "paths_on_same_lists": paths,
+            "rotate_with_neighbouring_host_ids_gbs": extra["contiguous_host"],
             "single_swaps": extra["singles"],
             "request_rotate_us": {"p50": M.percentile(extra["lat_us"], 0.5), "p99": M.percentile(extra["lat_us"], 0.99),
                                   "n": len(extra["lat_us"]),
@@ -394,6 +435,8 @@ def main() -> None:
     ap.add_argument("--path", type=int, default=0, help="KV_PATH_* (0 = auto)")
     ap.add_argument("--flags", type=int, default=0, help="KV_FLAG_* bits")
     ap.add_argument("--ctas", type=int, default=0, help="CTAs per direction (0 = default)")
+    ap.add_argument("--staging-mib", type=int, default=0, help="per-direction staging of the staged path (0 = library default)")
+    ap.add_argument("--quick", action="store_true", help="skip the per-segment comparator path")
     ap.add_argument("--small", action="store_true",
                     help="profiling case: same shape and kernels, 16 requests, 4 rotated each way, 6 GB + 8 GB pools")
     args = ap.parse_args()

@@ -53,7 +53,7 @@ extern "C" {
 #define KV_HOST_LAYER_FIRST   1
 
 /* transfer paths (how the host link is driven) */
-#define KV_PATH_AUTO          0     /* per-block-size choice measured on B200 (see kv_path_for)          */
+#define KV_PATH_AUTO          0     /* choice by bytes per block measured on B200 (see kv_path_for)      */
 #define KV_PATH_ZEROCOPY      1     /* SM kernels read/write mapped pinned host memory directly          */
 #define KV_PATH_STAGED        2     /* pack kernel -> contiguous HBM staging -> copy engine (and reverse)*/
 #define KV_PATH_CE2D          3     /* one strided 2-D copy-engine transfer per block, no kernel         */
@@ -66,6 +66,9 @@ extern "C" {
                                        bulk asynchronous copies through shared memory                    */
 #define KV_FLAG_FUSED_ROTATE    4   /* ZEROCOPY kv_rotate with disjoint lists: one launch, CTAs split
                                        between the directions, on the out stream                         */
+#define KV_FLAG_TIME_KERNELS    8   /* bracket every HBM-to-HBM gather / scatter kernel (STAGED pack / unpack,
+                                       kv_gather_blocks, kv_scatter_blocks) with events on its own stream;
+                                       kv_sync adds their durations to the timed_* statistics            */
 
 typedef struct kv_pool kv_pool_t;   /* opaque; owned by the library */
 
@@ -83,9 +86,12 @@ typedef struct {
     void   *stream_in;      /* likewise; must differ from stream_out for the directions to overlap        */
     int32_t path;           /* KV_PATH_* of the swap-out direction, and of swap-in unless path_in is set  */
     int32_t flags;          /* KV_FLAG_*                                                                  */
-    int32_t ctas_out;       /* CTAs of the swap-out kernel, 0 = default for the path                      */
+    int32_t ctas_out;       /* CTAs of the zero-copy swap-out kernel, 0 = 64                              */
     int32_t ctas_in;        /* CTAs of the swap-in kernel, 0 = default                                    */
-    int64_t staging_bytes;  /* per-direction HBM staging buffer of the STAGED path, 0 = 64 MiB            */
+    int64_t staging_bytes;  /* per-direction HBM staging of the STAGED path (two halves used as a double
+                               buffer, allocated at the first staged call); 0 = 2 GiB or a sixteenth of the
+                               device pool, whichever is smaller; at least 2*BLK.  Larger halves mean fewer
+                               and longer pack / unpack launches                                          */
     int32_t path_in;        /* KV_PATH_* of the swap-in direction; KV_PATH_AUTO (0) = same as `path`      */
     int32_t ce_streams;     /* streams per direction that the copy-engine paths spread their transfers
                                over (1..4), 0 = 1                                                         */
@@ -103,6 +109,9 @@ typedef struct {
     int32_t last_path_out, last_path_in;
     uint32_t device_status;            /* sticky bits written by kernels (0 = clean)                      */
     int32_t pad_;
+    double  timed_kernel_ms;           /* KV_FLAG_TIME_KERNELS: summed device time of the timed kernels   */
+    int64_t timed_kernel_bytes;        /* payload bytes those kernels moved (each read once, written once)*/
+    int64_t timed_kernels;             /* how many launches the two sums cover                            */
 } kv_stats_t;
 
 typedef struct {
@@ -150,6 +159,10 @@ int32_t kv_rotate(kv_pool_t *pool,
                   const int32_t *out_gpu, const int32_t *out_host, int64_t n_out,
                   const int32_t *in_host, const int32_t *in_gpu, int64_t n_in);
 
+/* Wait for outstanding work, then change the transfer path of each direction (KV_PATH_*; AUTO
+ * re-applies the rule of kv_path_for).  Pool contents are unaffected. */
+int32_t kv_pool_set_path(kv_pool_t *pool, int32_t path_out, int32_t path_in);
+
 /* Wait for both directions.  Returns KV_OK, or the first sticky asynchronous error
  * (KV_ERR_CUDA, KV_ERR_TIMEOUT).  Fills the last_* timing fields of the statistics. */
 int32_t kv_sync(kv_pool_t *pool);
@@ -178,8 +191,8 @@ const char *kv_last_error(kv_pool_t *pool);
 int64_t kv_seg_bytes(int32_t block_size, int32_t kv_heads, int32_t head_dim);
 int64_t kv_blk_bytes(int32_t num_layers, int32_t block_size, int32_t kv_heads, int32_t head_dim);
 
-/* The path KV_PATH_AUTO resolves to for a segment size. */
-int32_t kv_path_for(int64_t seg_bytes);
+/* The path KV_PATH_AUTO resolves to for a block of blk_bytes (= kv_blk_bytes of the shape). */
+int32_t kv_path_for(int64_t blk_bytes);
 
 /*
  * Host-link roofline probe (the analogue of the paper's appendix B bandwidth measurement, done
@@ -188,6 +201,24 @@ int32_t kv_path_for(int64_t seg_bytes);
  * its own pinned and device buffers.
  */
 int32_t kv_probe_link(int32_t device_id, int64_t bytes, int32_t reps, kv_link_probe_t *out);
+
+/*
+ * The same probe with the shape of the transfers as parameters: the bandwidth-versus-transfer-size
+ * curve of the paper's motivation study (the figure of section 3.2 on full-duplex bandwidth against
+ * segment size, and the launch-versus-transfer-time figure of section 4.3.1).  Each round issues
+ * total_bytes/copy_bytes copy-engine transfers of copy_bytes back to back on one stream per direction.
+ * rows <= 1: plain transfers.  rows > 1: strided 2-D transfers of `rows` rows of copy_bytes/rows bytes,
+ * row r at start + r*host_pitch on the host and start + r*dev_pitch on the device (0 = rows packed).
+ * The transfers start at consecutive places of span_bytes-sized buffers (wrapping), or at seeded
+ * pseudo-random row-aligned offsets when scattered != 0.  One warm-up round, then `rounds` timed
+ * ones; the best is kept.  out->bytes = copy_bytes, out->reps = transfers per round.
+ */
+typedef struct {
+    int64_t copy_bytes, total_bytes, span_bytes;
+    int32_t scattered, rounds;
+    int64_t rows, host_pitch, dev_pitch;
+} kv_probe_spec_t;
+int32_t kv_probe_link_ex(int32_t device_id, const kv_probe_spec_t *spec, kv_link_probe_t *out);
 
 #ifdef __cplusplus
 }

@@ -37,6 +37,7 @@ PATH_NAMES = {0: "auto", 1: "zerocopy", 2: "staged", 3: "ce2d", 4: "naive"}
 KV_FLAG_ALLOW_OVERLAP = 1
 KV_FLAG_LDST_KERNEL = 2
 KV_FLAG_FUSED_ROTATE = 4
+KV_FLAG_TIME_KERNELS = 8
 
 
 class kv_pool_config_t(C.Structure):
@@ -53,7 +54,8 @@ class kv_stats_t(C.Structure):
                 ("calls_in", C.c_int64), ("kernel_launches", C.c_int64), ("ce_copies", C.c_int64),
                 ("last_out_ms", C.c_double), ("last_in_ms", C.c_double), ("last_union_ms", C.c_double),
                 ("last_path_out", C.c_int32), ("last_path_in", C.c_int32),
-                ("device_status", C.c_uint32), ("pad_", C.c_int32)]
+                ("device_status", C.c_uint32), ("pad_", C.c_int32),
+                ("timed_kernel_ms", C.c_double), ("timed_kernel_bytes", C.c_int64), ("timed_kernels", C.c_int64)]
 
 
 class kv_link_probe_t(C.Structure):
@@ -62,9 +64,15 @@ class kv_link_probe_t(C.Structure):
                 ("reps", C.c_int32), ("pad_", C.c_int32)]
 
 
-EXPORTS = ["kv_pool_create", "kv_pool_destroy", "kv_swap_out", "kv_swap_in", "kv_rotate", "kv_sync",
+class kv_probe_spec_t(C.Structure):
+    _fields_ = [("copy_bytes", C.c_int64), ("total_bytes", C.c_int64), ("span_bytes", C.c_int64),
+                ("scattered", C.c_int32), ("rounds", C.c_int32),
+                ("rows", C.c_int64), ("host_pitch", C.c_int64), ("dev_pitch", C.c_int64)]
+
+
+EXPORTS = ["kv_pool_create", "kv_pool_destroy", "kv_pool_set_path", "kv_swap_out", "kv_swap_in", "kv_rotate", "kv_sync",
            "kv_gather_blocks", "kv_scatter_blocks", "kv_host_ptr", "kv_get_stats", "kv_last_error",
-           "kv_seg_bytes", "kv_blk_bytes", "kv_path_for", "kv_probe_link"]
+           "kv_seg_bytes", "kv_blk_bytes", "kv_path_for", "kv_probe_link", "kv_probe_link_ex"]
 
 _lib = None
 
@@ -89,6 +97,8 @@ def lib() -> C.CDLL:
     L.kv_rotate.argtypes = [vp, i32p, i32p, i64, i32p, i32p, i64]
     L.kv_sync.restype = C.c_int32
     L.kv_sync.argtypes = [vp]
+    L.kv_pool_set_path.restype = C.c_int32
+    L.kv_pool_set_path.argtypes = [vp, C.c_int32, C.c_int32]
     L.kv_gather_blocks.restype = C.c_int32
     L.kv_gather_blocks.argtypes = [vp, i32p, i64, vp]
     L.kv_scatter_blocks.restype = C.c_int32
@@ -107,6 +117,8 @@ def lib() -> C.CDLL:
     L.kv_path_for.argtypes = [i64]
     L.kv_probe_link.restype = C.c_int32
     L.kv_probe_link.argtypes = [C.c_int32, i64, C.c_int32, C.POINTER(kv_link_probe_t)]
+    L.kv_probe_link_ex.restype = C.c_int32
+    L.kv_probe_link_ex.argtypes = [C.c_int32, C.POINTER(kv_probe_spec_t), C.POINTER(kv_link_probe_t)]
     _lib = L
     return L
 
@@ -134,13 +146,24 @@ def kv_blk_bytes(num_layers: int, block_size: int, kv_heads: int, head_dim: int)
     return lib().kv_blk_bytes(num_layers, block_size, kv_heads, head_dim)
 
 
-def kv_path_for(seg_bytes: int) -> int:
-    return lib().kv_path_for(seg_bytes)
+def kv_path_for(blk_bytes: int) -> int:
+    return lib().kv_path_for(blk_bytes)
 
 
 def kv_probe_link(device_id: int = 0, nbytes: int = 256 << 20, reps: int = 4) -> dict:
     out = kv_link_probe_t()
     rc = lib().kv_probe_link(device_id, nbytes, reps, C.byref(out))
+    if rc != KV_OK:
+        raise KVError(rc, lib().kv_last_error(None).decode())
+    return {k: getattr(out, k) for k, _ in kv_link_probe_t._fields_ if k != "pad_"}
+
+
+def kv_probe_link_ex(device_id: int, copy_bytes: int, total_bytes: int, span_bytes: int,
+                     scattered: bool = False, rounds: int = 3, rows: int = 1, host_pitch: int = 0,
+                     dev_pitch: int = 0) -> dict:
+    spec = kv_probe_spec_t(copy_bytes, total_bytes, span_bytes, int(scattered), rounds, rows, host_pitch, dev_pitch)
+    out = kv_link_probe_t()
+    rc = lib().kv_probe_link_ex(device_id, C.byref(spec), C.byref(out))
     if rc != KV_OK:
         raise KVError(rc, lib().kv_last_error(None).decode())
     return {k: getattr(out, k) for k, _ in kv_link_probe_t._fields_ if k != "pad_"}
@@ -217,6 +240,9 @@ class KVPool:
     def kv_rotate_raw(self, ogp, ohp, n_out, ihp, igp, n_in) -> int:
         """Same call with pre-marshalled ``POINTER(c_int32)`` arguments (for timing loops)."""
         return lib().kv_rotate(self._h, ogp, ohp, n_out, ihp, igp, n_in)
+
+    def kv_pool_set_path(self, path_out: int, path_in: int, check: bool = True) -> int:
+        return self._ret(lib().kv_pool_set_path(self._h, path_out, path_in), check)
 
     def kv_sync(self, check: bool = True) -> int:
         return self._ret(lib().kv_sync(self._h), check)

@@ -29,6 +29,18 @@ constexpr int LDST_CHUNK = LDST_THREADS * LDST_UNROLL * 16;
 
 thread_local char g_err[256] = "";
 
+// One copy-engine transfer of the STAGED path: `rows` rows of `width` bytes, packed back to back in
+// the staging half, `host_pitch` bytes apart on the host (rows == 1: a plain transfer).
+struct CeOp {
+    int64_t host_off, stage_off, width, host_pitch;
+    int32_t rows;
+};
+// Sorted list positions [lo, hi) go through one staging half; ops [op_lo, op_hi) move them.
+struct CeChunk {
+    int64_t lo, hi;
+    int32_t op_lo, op_hi;
+};
+
 struct DirState {
     cudaStream_t stream = nullptr;
     bool owns_stream = false;
@@ -38,7 +50,21 @@ struct DirState {
     cudaEvent_t ev_end[KV_SLOTS] = {};
     uint64_t issued = 0;               // calls issued on this direction (sequence number of the latest)
     uint64_t done = 0;                 // latest call known to be complete
-    uint8_t *stage = nullptr;          // HBM staging (STAGED path), allocated on first use
+    // STAGED path: two staging halves in HBM (allocated on first use) worked as a double buffer: the
+    // pack/unpack kernels run on `kstream`, the copy-engine transfers on `stream`
+    uint8_t *stage = nullptr;
+    int64_t half_blocks = 0;           // blocks per half
+    cudaStream_t kstream = nullptr;
+    cudaEvent_t kfork_ev = nullptr;
+    cudaEvent_t ev_a[2] = {};          // half filled   (out: packed by the kernel;   in: landed from the host)
+    cudaEvent_t ev_b[2] = {};          // half drained  (out: copied to the host;     in: scattered by the kernel)
+    // optional timing of the pack / unpack kernels (KV_FLAG_TIME_KERNELS): event pairs on kstream
+    std::vector<cudaEvent_t> kev;
+    std::vector<int64_t> kev_bytes;
+    int kev_used = 0;
+    std::vector<int32_t> order;        // list positions sorted by host id
+    std::vector<CeOp> ops;             // transfers of the current call, in issue order
+    std::vector<CeChunk> chunks;       // the call cut into staging-half-sized pieces
     int ctas = 0;
     int path = 0;                      // configured path of this direction (may be KV_PATH_AUTO)
     // copy-engine paths spread their transfers over nsub streams: sub[0] is `stream`, the others
@@ -61,6 +87,7 @@ struct kv_pool {
     uint8_t *host_dev = nullptr;       // the same memory as the device sees it
     bool owns_host = false, registered_host = false;
     int sm_count = 0;
+    int64_t max_pitch = 0;             // largest row pitch a 2-D copy-engine transfer accepts
     DirState dir[2];                   // 0 = out, 1 = in
     unsigned int *status_host = nullptr, *status_dev = nullptr;   // mapped pinned status word
     // per-block bookkeeping for validation and cross-direction ordering
@@ -144,6 +171,34 @@ cudaError_t launch_job(kv_pool *p, const KvJob &job, cudaStream_t stream)
     }
     p->stats.kernel_launches++;
     return cudaGetLastError();
+}
+
+constexpr int KV_MAX_TIMED = 2048;     // kernel launches per direction timed between two kv_sync calls
+
+// HBM-to-HBM gather / scatter launch, bracketed by events on its stream when kernel timing is on
+cudaError_t launch_timed(kv_pool *p, DirState &s, cudaStream_t stream, const KvJob &job, int64_t payload_bytes)
+{
+    const bool timed = (p->cfg.flags & KV_FLAG_TIME_KERNELS) && s.kev_used < KV_MAX_TIMED;
+    if (timed) {
+        while ((int)s.kev.size() < 2 * (s.kev_used + 1)) {
+            cudaEvent_t e;
+            cudaError_t rc = cudaEventCreate(&e);
+            if (rc != cudaSuccess) return rc;
+            s.kev.push_back(e);
+        }
+        if ((int)s.kev_bytes.size() <= s.kev_used) s.kev_bytes.resize((size_t)s.kev_used + 1);
+        cudaError_t rc = cudaEventRecord(s.kev[2 * (size_t)s.kev_used], stream);
+        if (rc != cudaSuccess) return rc;
+    }
+    cudaError_t rc = launch_job(p, job, stream);
+    if (rc != cudaSuccess) return rc;
+    if (timed) {
+        rc = cudaEventRecord(s.kev[2 * (size_t)s.kev_used + 1], stream);
+        if (rc != cudaSuccess) return rc;
+        s.kev_bytes[(size_t)s.kev_used] = payload_bytes;
+        s.kev_used++;
+    }
+    return cudaSuccess;
 }
 
 // ---------------------------------------------------------------------------------------------
@@ -233,7 +288,8 @@ struct DirCall {
     int path;
     // copy-engine issue state (CE paths are issued in slices so the two directions interleave)
     int64_t ce_next = 0;
-    int64_t chunk_lo = 0;
+    int chunk_idx = 0;                 // STAGED: chunk being issued, next op of it
+    int op_next = 0;
     bool chunk_open = false;
     unsigned rr = 0;                   // round-robin cursor over the direction's CE streams
 };
@@ -241,7 +297,7 @@ struct DirCall {
 int resolve_path(const kv_pool *p, int d)
 {
     int path = p->dir[d].path;
-    if (path == KV_PATH_AUTO) path = kv_path_for(p->seg);
+    if (path == KV_PATH_AUTO) path = kv_path_for(p->blk);
     return path;
 }
 
@@ -264,6 +320,70 @@ int32_t ce_join(kv_pool *p, DirState &s)
     return KV_OK;
 }
 
+// STAGED path, host side of one direction of one call: sort the pairs by host id so that blocks that
+// are neighbours in host memory become one transfer, cut the sorted list into staging-half-sized
+// chunks, and turn every chunk into as few copy-engine transfers as its host ids allow.
+//   - a run of consecutive host ids is one plain transfer;
+//   - runs of equal length whose starts are equally spaced become one strided 2-D transfer (any two
+//     runs are "equally spaced", so isolated blocks still travel two per transfer).
+// The cost of a transfer on the copy engine is a fixed start-up plus its bytes, so fewer and larger
+// transfers are what keeps the link busy.
+int32_t plan_staged(kv_pool *p, DirCall &c)
+{
+    DirState &s = p->dir[c.d];
+    const bool layer_first = p->cfg.host_layout == KV_HOST_LAYER_FIRST;
+    try {
+        s.order.resize((size_t)c.n);
+        for (int64_t i = 0; i < c.n; ++i) s.order[(size_t)i] = (int32_t)i;
+        if (!layer_first)
+            std::sort(s.order.begin(), s.order.end(), [&](int32_t a, int32_t b) { return c.host_ids[a] < c.host_ids[b]; });
+        s.ops.clear();
+        s.chunks.clear();
+        // The first chunk of a swap-out is half as long as the rest: its first transfer starts sooner, and
+        // in a rotation the pack kernels then run midway between the swap-in's unpack kernels instead of
+        // at the same moments (both directions advance one chunk per equal stretch of link time).
+        const int64_t first = (c.d == 0 && c.n > s.half_blocks) ? std::max<int64_t>(1, s.half_blocks / 2) : s.half_blocks;
+        for (int64_t lo = 0, hi = 0; lo < c.n; lo = hi) {
+            hi = std::min(c.n, lo + (lo == 0 ? first : s.half_blocks));
+            CeChunk ch{lo, hi, (int32_t)s.ops.size(), 0};
+            if (layer_first) {
+                // one strided transfer per block: `planes` rows of SEG bytes, a whole host plane apart
+                for (int64_t k = lo; k < hi; ++k)
+                    s.ops.push_back(CeOp{(int64_t)c.host_ids[s.order[(size_t)k]] * p->seg, (k - lo) * p->blk, p->seg,
+                                         p->cfg.num_host_blocks * p->seg, p->planes});
+            } else {
+                int64_t k = lo;
+                auto hid = [&](int64_t q) { return (int64_t)c.host_ids[s.order[(size_t)q]]; };
+                auto run_len = [&](int64_t q) {
+                    int64_t r = 1;
+                    while (q + r < hi && hid(q + r) == hid(q) + r) ++r;
+                    return r;
+                };
+                while (k < hi) {
+                    const int64_t r = run_len(k);
+                    CeOp op{hid(k) * p->blk, (k - lo) * p->blk, r * p->blk, r * p->blk, 1};
+                    int64_t nxt = k + r;
+                    // further runs of the same length at a constant spacing join as extra rows
+                    while (nxt < hi && run_len(nxt) == r) {
+                        const int64_t pitch = (hid(nxt) - hid(nxt - r)) * p->blk;
+                        if (pitch < op.width || pitch > p->max_pitch || (op.rows > 1 && pitch != op.host_pitch)) break;
+                        op.host_pitch = pitch;
+                        op.rows++;
+                        nxt += r;
+                    }
+                    s.ops.push_back(op);
+                    k = nxt;
+                }
+            }
+            ch.op_hi = (int32_t)s.ops.size();
+            s.chunks.push_back(ch);
+        }
+    } catch (...) {
+        return fail(p, KV_ERR_NOMEM, "out of host memory");
+    }
+    return KV_OK;
+}
+
 int32_t begin_dir(kv_pool *p, DirCall &c, bool wait_other)
 {
     DirState &s = p->dir[c.d];
@@ -274,9 +394,26 @@ int32_t begin_dir(kv_pool *p, DirCall &c, bool wait_other)
     c.pairs_dev = s.ring_dev + (size_t)c.slot * 2 * p->cap;
     c.aux_host = c.pairs_host + p->cap;
     c.aux_dev = c.pairs_dev + p->cap;
-    for (int64_t i = 0; i < c.n; ++i) {
-        c.pairs_host[i] = (c.d == 0) ? make_int2(c.gpu_ids[i], c.host_ids[i]) : make_int2(c.host_ids[i], c.gpu_ids[i]);
-        c.aux_host[i] = (c.d == 0) ? make_int2(c.gpu_ids[i], (int)i) : make_int2((int)i, c.gpu_ids[i]);
+    if (c.path == KV_PATH_STAGED) {
+        if (!s.stage) {
+            s.half_blocks = std::max<int64_t>(1, p->cfg.staging_bytes / 2 / p->blk);
+            cudaError_t e = cudaMalloc((void **)&s.stage, (size_t)(2 * s.half_blocks * p->blk));
+            if (e != cudaSuccess) {
+                s.stage = nullptr;
+                (void)cudaGetLastError();
+                return fail(p, KV_ERR_NOMEM, "staging buffer allocation failed");
+            }
+        }
+        int32_t rc = plan_staged(p, c);
+        if (rc != KV_OK) return rc;
+        // the kernel sees (device block id, position in the sorted list)
+        for (int64_t k = 0; k < c.n; ++k) {
+            const int32_t g = c.gpu_ids[s.order[(size_t)k]];
+            c.aux_host[k] = (c.d == 0) ? make_int2(g, (int)k) : make_int2((int)k, g);
+        }
+    } else if (c.path == KV_PATH_ZEROCOPY) {
+        for (int64_t i = 0; i < c.n; ++i)
+            c.pairs_host[i] = (c.d == 0) ? make_int2(c.gpu_ids[i], c.host_ids[i]) : make_int2(c.host_ids[i], c.gpu_ids[i]);
     }
     if (wait_other) {
         DirState &o = p->dir[1 - c.d];
@@ -287,14 +424,9 @@ int32_t begin_dir(kv_pool *p, DirCall &c, bool wait_other)
         KV_CUDA(p, cudaMemcpyAsync(c.pairs_dev, c.pairs_host, (size_t)c.n * sizeof(int2), cudaMemcpyHostToDevice, s.stream));
     } else if (c.path == KV_PATH_STAGED) {
         KV_CUDA(p, cudaMemcpyAsync(c.aux_dev, c.aux_host, (size_t)c.n * sizeof(int2), cudaMemcpyHostToDevice, s.stream));
-        if (!s.stage) {
-            cudaError_t e = cudaMalloc((void **)&s.stage, (size_t)p->cfg.staging_bytes);
-            if (e != cudaSuccess) {
-                s.stage = nullptr;
-                (void)cudaGetLastError();
-                return fail(p, KV_ERR_NOMEM, "staging buffer allocation failed");
-            }
-        }
+        // the kernel stream starts after everything issued so far on this direction
+        KV_CUDA(p, cudaEventRecord(s.kfork_ev, s.stream));
+        KV_CUDA(p, cudaStreamWaitEvent(s.kstream, s.kfork_ev, 0));
     }
     if (c.path == KV_PATH_CE2D || c.path == KV_PATH_NAIVE) {
         int32_t rc = ce_fork(p, s);
@@ -311,6 +443,11 @@ int32_t end_dir(kv_pool *p, DirCall &c)
     if (c.path == KV_PATH_CE2D || c.path == KV_PATH_NAIVE) {
         int32_t rc = ce_join(p, s);
         if (rc != KV_OK) return rc;
+    }
+    if (c.path == KV_PATH_STAGED && c.d == 1) {
+        // the call ends when the last unpack kernels have run (they are on the kernel stream)
+        const int nch = (int)s.chunks.size();
+        for (int q = std::max(0, nch - 2); q < nch; ++q) KV_CUDA(p, cudaStreamWaitEvent(s.stream, s.ev_b[q & 1], 0));
     }
     KV_CUDA(p, cudaEventRecord(s.ev_end[c.slot], s.stream));
     const int64_t bytes = c.n * p->blk;
@@ -386,60 +523,65 @@ int32_t ce_issue_some(kv_pool *p, DirCall &c, int budget, bool &finished)
         finished = c.ce_next >= c.n;
         return KV_OK;
     }
-    // STAGED: the list is cut into chunks of at most stage_blocks blocks.  Out: gather kernel into the
-    // staging buffer, then one transfer per run of consecutive host ids.  In: the transfers, then the
-    // scatter kernel.  Everything of one direction is on one stream, so reuse of the buffer is ordered.
-    const int64_t stage_blocks = std::max<int64_t>(1, p->cfg.staging_bytes / p->blk);
-    while (budget > 0 && c.chunk_lo < c.n) {
-        const int64_t lo = c.chunk_lo, hi = std::min(c.n, lo + stage_blocks);
+    // STAGED: chunk q of the sorted list goes through staging half q & 1.
+    //   out: kernel stream packs the half, then the transfers drain it on the direction's stream;
+    //   in:  the transfers fill the half, then the kernel stream unpacks it.
+    // While one half is on the link the other is being packed / unpacked.
+    while (budget > 0 && c.chunk_idx < (int)s.chunks.size()) {
+        const CeChunk &ch = s.chunks[(size_t)c.chunk_idx];
+        const int b = c.chunk_idx & 1;
+        uint8_t *half = s.stage + (size_t)b * (size_t)(s.half_blocks * p->blk);
         KvJob job;
         fill_geometry(p, job);
         job.dir[1] = KvDir{};
         KvDir &kd = job.dir[0];
-        // staging block of list position k is at stage + (k - lo)*BLK
-        const KvSide st = packed_side(p, s.stage - lo * p->blk);
+        // the staging slot of sorted position k is half + (k - lo)*BLK
+        const KvSide st = packed_side(p, half - ch.lo * p->blk);
         kd.src = (c.d == 0) ? device_side(p) : st;
         kd.dst = (c.d == 0) ? st : device_side(p);
-        kd.pairs = c.aux_dev + lo;
-        kd.n = (int)(hi - lo);
+        kd.pairs = c.aux_dev + ch.lo;
+        kd.n = (int)(ch.hi - ch.lo);
         kd.ctas = clamp_ctas(job, kd, p->sm_count);
-        if (c.ce_next == lo && !c.chunk_open) {
-            // out: gather into the staging buffer first; both: the extra streams start after what
-            // the main stream has done so far (the gather, or the previous chunk's scatter)
-            if (c.d == 0) KV_CUDA(p, launch_job(p, job, s.stream));
-            int32_t rc = ce_fork(p, s);
-            if (rc != KV_OK) return rc;
+        if (!c.chunk_open) {
+            if (c.d == 0) {
+                if (c.chunk_idx >= 2) KV_CUDA(p, cudaStreamWaitEvent(s.kstream, s.ev_b[b], 0));
+                KV_CUDA(p, launch_timed(p, s, s.kstream, job, (ch.hi - ch.lo) * p->blk));
+                KV_CUDA(p, cudaEventRecord(s.ev_a[b], s.kstream));
+                KV_CUDA(p, cudaStreamWaitEvent(s.stream, s.ev_a[b], 0));
+            } else if (c.chunk_idx >= 2) {
+                KV_CUDA(p, cudaStreamWaitEvent(s.stream, s.ev_b[b], 0));
+            }
             c.chunk_open = true;
+            c.op_next = ch.op_lo;
         }
-        while (budget > 0 && c.ce_next < hi) {
-            int64_t k = c.ce_next, run = 1;
-            if (p->cfg.host_layout == KV_HOST_BLOCK_FIRST) {
-                while (k + run < hi && c.host_ids[k + run] == c.host_ids[k] + run) ++run;
-                uint8_t *hv = host_block_ptr(p, c.host_ids[k]);
-                uint8_t *sv = s.stage + (k - lo) * p->blk;
-                KV_CUDA(p, cudaMemcpyAsync(c.d == 0 ? hv : sv, c.d == 0 ? sv : hv, (size_t)(run * p->blk), kind, s.sub[c.rr++ % s.nsub]));
+        while (budget > 0 && c.op_next < ch.op_hi) {
+            const CeOp &op = s.ops[(size_t)c.op_next];
+            uint8_t *hv = p->host + op.host_off, *sv = half + op.stage_off;
+            if (op.rows == 1) {
+                KV_CUDA(p, cudaMemcpyAsync(c.d == 0 ? hv : sv, c.d == 0 ? sv : hv, (size_t)op.width, kind, s.stream));
+            } else if (c.d == 0) {
+                KV_CUDA(p, cudaMemcpy2DAsync(hv, (size_t)op.host_pitch, sv, (size_t)op.width, (size_t)op.width, (size_t)op.rows, kind, s.stream));
             } else {
-                uint8_t *hv = host_block_ptr(p, c.host_ids[k]);
-                uint8_t *sv = s.stage + (k - lo) * p->blk;
-                cudaStream_t cs = s.sub[c.rr++ % s.nsub];
-                if (c.d == 0)
-                    KV_CUDA(p, cudaMemcpy2DAsync(hv, host_pitch(p), sv, (size_t)p->seg, (size_t)p->seg, (size_t)p->planes, kind, cs));
-                else
-                    KV_CUDA(p, cudaMemcpy2DAsync(sv, (size_t)p->seg, hv, host_pitch(p), (size_t)p->seg, (size_t)p->planes, kind, cs));
+                KV_CUDA(p, cudaMemcpy2DAsync(sv, (size_t)op.width, hv, (size_t)op.host_pitch, (size_t)op.width, (size_t)op.rows, kind, s.stream));
             }
             p->stats.ce_copies++;
-            c.ce_next += run;
+            c.op_next++;
             --budget;
         }
-        if (c.ce_next >= hi) {
-            int32_t rc = ce_join(p, s);
-            if (rc != KV_OK) return rc;
-            if (c.d == 1) KV_CUDA(p, launch_job(p, job, s.stream));
-            c.chunk_lo = hi;
+        if (c.op_next >= ch.op_hi) {
+            if (c.d == 0) {
+                KV_CUDA(p, cudaEventRecord(s.ev_b[b], s.stream));
+            } else {
+                KV_CUDA(p, cudaEventRecord(s.ev_a[b], s.stream));
+                KV_CUDA(p, cudaStreamWaitEvent(s.kstream, s.ev_a[b], 0));
+                KV_CUDA(p, launch_timed(p, s, s.kstream, job, (ch.hi - ch.lo) * p->blk));
+                KV_CUDA(p, cudaEventRecord(s.ev_b[b], s.kstream));
+            }
+            c.chunk_idx++;
             c.chunk_open = false;
         }
     }
-    finished = c.chunk_lo >= c.n;
+    finished = c.chunk_idx >= (int)s.chunks.size();
     return KV_OK;
 }
 
@@ -538,10 +680,13 @@ int64_t kv_blk_bytes(int32_t num_layers, int32_t block_size, int32_t kv_heads, i
     return 2 * (int64_t)num_layers * kv_seg_bytes(block_size, kv_heads, head_dim);
 }
 
-int32_t kv_path_for(int64_t seg_bytes)
+int32_t kv_path_for(int64_t blk_bytes)
 {
-    (void)seg_bytes;
-    return KV_PATH_ZEROCOPY;
+    // Measured on B200 behind PCIe Gen5 x16, both directions busy, scattered ids: a copy-engine
+    // transfer costs a fixed start-up (about 10 us with the other direction busy) plus its bytes, so
+    // the staged path wins once its transfers (two blocks each when no host ids are neighbours) carry
+    // 4 MiB or more; below that the zero-copy kernels, which pay no per-block cost, are ahead.
+    return blk_bytes >= (2ll << 20) ? KV_PATH_STAGED : KV_PATH_ZEROCOPY;
 }
 
 const char *kv_last_error(kv_pool_t *pool) { return pool ? pool->err : g_err; }
@@ -581,8 +726,9 @@ int32_t kv_pool_create(const kv_pool_config_t *cfg, kv_pool_t **out)
     p->dev = (uint8_t *)cfg->device_base;
     p->err[0] = 0;
     memset(&p->stats, 0, sizeof(p->stats));
-    if (p->cfg.staging_bytes == 0) p->cfg.staging_bytes = 64ll << 20;
-    if (p->cfg.staging_bytes < blk) p->cfg.staging_bytes = blk;
+    // default staging: 2 GiB per direction, but no more than a sixteenth of the device pool
+    if (p->cfg.staging_bytes == 0) p->cfg.staging_bytes = std::min<int64_t>(2ll << 30, cfg->num_gpu_blocks * blk / 16);
+    if (p->cfg.staging_bytes < 2 * blk) p->cfg.staging_bytes = 2 * blk;
 
 #define KV_CREATE_CUDA(expr)                                   \
     do {                                                       \
@@ -597,6 +743,7 @@ int32_t kv_pool_create(const kv_pool_config_t *cfg, kv_pool_t **out)
     cudaDeviceProp prop;
     KV_CREATE_CUDA(cudaGetDeviceProperties(&prop, cfg->device_id));
     p->sm_count = prop.multiProcessorCount;
+    p->max_pitch = (int64_t)std::min<size_t>(prop.memPitch, (size_t)INT32_MAX);
 
     const size_t host_bytes = (size_t)cfg->num_host_blocks * (size_t)blk;
     if (cfg->host_base) {
@@ -642,11 +789,17 @@ int32_t kv_pool_create(const kv_pool_config_t *cfg, kv_pool_t **out)
             KV_CREATE_CUDA(cudaEventCreate(&s.ev_start[k]));
             KV_CREATE_CUDA(cudaEventCreate(&s.ev_end[k]));
         }
-        s.ctas = want_ctas[d] > 0 ? want_ctas[d] : 32;
+        s.ctas = want_ctas[d] > 0 ? want_ctas[d] : 64;
         s.path = (d == 1 && cfg->path_in != KV_PATH_AUTO) ? cfg->path_in : cfg->path;
         s.nsub = cfg->ce_streams > 0 ? cfg->ce_streams : 1;
         s.sub[0] = s.stream;
         KV_CREATE_CUDA(cudaEventCreateWithFlags(&s.fork_ev, cudaEventDisableTiming));
+        KV_CREATE_CUDA(cudaStreamCreateWithFlags(&s.kstream, cudaStreamNonBlocking));
+        KV_CREATE_CUDA(cudaEventCreateWithFlags(&s.kfork_ev, cudaEventDisableTiming));
+        for (int k = 0; k < 2; ++k) {
+            KV_CREATE_CUDA(cudaEventCreateWithFlags(&s.ev_a[k], cudaEventDisableTiming));
+            KV_CREATE_CUDA(cudaEventCreateWithFlags(&s.ev_b[k], cudaEventDisableTiming));
+        }
         for (int k = 1; k < s.nsub; ++k) {
             KV_CREATE_CUDA(cudaStreamCreateWithFlags(&s.sub[k], cudaStreamNonBlocking));
             KV_CREATE_CUDA(cudaEventCreateWithFlags(&s.join_ev[k], cudaEventDisableTiming));
@@ -690,6 +843,16 @@ int32_t kv_pool_destroy(kv_pool_t *p)
             if (s.join_ev[k]) (void)cudaEventDestroy(s.join_ev[k]);
         }
         if (s.fork_ev) (void)cudaEventDestroy(s.fork_ev);
+        if (s.kstream) {
+            (void)cudaStreamSynchronize(s.kstream);
+            (void)cudaStreamDestroy(s.kstream);
+        }
+        if (s.kfork_ev) (void)cudaEventDestroy(s.kfork_ev);
+        for (cudaEvent_t e : s.kev) (void)cudaEventDestroy(e);
+        for (int k = 0; k < 2; ++k) {
+            if (s.ev_a[k]) (void)cudaEventDestroy(s.ev_a[k]);
+            if (s.ev_b[k]) (void)cudaEventDestroy(s.ev_b[k]);
+        }
         if (s.ring_host) (void)cudaFreeHost(s.ring_host);
         if (s.ring_dev) (void)cudaFree(s.ring_dev);
         if (s.stage) (void)cudaFree(s.stage);
@@ -816,6 +979,18 @@ int32_t kv_rotate(kv_pool_t *p, const int32_t *out_gpu, const int32_t *out_host,
     return rc;
 }
 
+int32_t kv_pool_set_path(kv_pool_t *p, int32_t path_out, int32_t path_in)
+{
+    if (!p) return KV_ERR_INVALID_ARG;
+    if (path_out < KV_PATH_AUTO || path_out > KV_PATH_NAIVE || path_in < KV_PATH_AUTO || path_in > KV_PATH_NAIVE)
+        return fail(p, KV_ERR_INVALID_ARG, "unknown path");
+    int32_t rc = kv_sync(p);
+    if (rc != KV_OK) return rc;
+    p->dir[0].path = path_out;
+    p->dir[1].path = path_in;
+    return KV_OK;
+}
+
 int32_t kv_sync(kv_pool_t *p)
 {
     if (!p) return KV_ERR_INVALID_ARG;
@@ -845,6 +1020,19 @@ int32_t kv_sync(kv_pool_t *p)
         (void)cudaGetLastError();
         p->union_valid = false;
     }
+    for (int d = 0; d < 2; ++d) {
+        DirState &s = p->dir[d];
+        for (int k = 0; k < s.kev_used; ++k) {
+            float ms = 0.f;
+            if (cudaEventElapsedTime(&ms, s.kev[2 * (size_t)k], s.kev[2 * (size_t)k + 1]) == cudaSuccess) {
+                p->stats.timed_kernel_ms += ms;
+                p->stats.timed_kernel_bytes += s.kev_bytes[(size_t)k];
+                p->stats.timed_kernels++;
+            }
+        }
+        s.kev_used = 0;
+    }
+    (void)cudaGetLastError();
     const unsigned int st = *(volatile unsigned int *)p->status_host;
     p->stats.device_status = st;
     if (st & KV_DEV_TIMEOUT) {
@@ -887,7 +1075,7 @@ static int32_t device_leg(kv_pool_t *p, const int32_t *gpu_ids, int64_t n, const
     kd.n = (int)n;
     const int want = (d == 0 ? p->cfg.ctas_out : p->cfg.ctas_in);
     kd.ctas = clamp_ctas(job, kd, want > 0 ? want : p->sm_count);
-    KV_CUDA(p, launch_job(p, job, s.stream));
+    KV_CUDA(p, launch_timed(p, s, s.stream, job, n * p->blk));
     KV_CUDA(p, cudaEventRecord(s.ev_end[slot], s.stream));
     s.issued = seq;
     p->union_slot[d] = slot;
@@ -922,11 +1110,47 @@ int32_t kv_get_stats(kv_pool_t *p, kv_stats_t *st)
     return KV_OK;
 }
 
-int32_t kv_probe_link(int32_t device_id, int64_t bytes, int32_t reps, kv_link_probe_t *out)
+int32_t kv_probe_link_ex(int32_t device_id, const kv_probe_spec_t *spec, kv_link_probe_t *out)
 {
-    if (!out || bytes <= 0 || reps <= 0) return fail(nullptr, KV_ERR_INVALID_ARG, "bad probe arguments");
+    if (!out || !spec || spec->copy_bytes <= 0 || spec->total_bytes < spec->copy_bytes || spec->rounds <= 0 || spec->rows < 0)
+        return fail(nullptr, KV_ERR_INVALID_ARG, "bad probe arguments");
+    const int64_t rows = spec->rows > 1 ? spec->rows : 1;
+    if (spec->copy_bytes % rows) return fail(nullptr, KV_ERR_INVALID_ARG, "copy_bytes must be a multiple of rows");
+    const size_t width = (size_t)(spec->copy_bytes / rows);
+    const size_t hpitch = spec->host_pitch > 0 ? (size_t)spec->host_pitch : width;
+    const size_t dpitch = spec->dev_pitch > 0 ? (size_t)spec->dev_pitch : width;
+    if (hpitch < width || dpitch < width) return fail(nullptr, KV_ERR_INVALID_ARG, "pitch smaller than a row");
+    // bytes from the first byte of a transfer to its last, on each side
+    const size_t foot_h = (size_t)(rows - 1) * hpitch + width, foot_d = (size_t)(rows - 1) * dpitch + width;
+    if ((size_t)spec->span_bytes < foot_h || (size_t)spec->span_bytes < foot_d)
+        return fail(nullptr, KV_ERR_INVALID_ARG, "span_bytes smaller than one transfer's footprint");
     memset(out, 0, sizeof(*out));
     KV_CUDA(nullptr, cudaSetDevice(device_id));
+    const size_t span = (size_t)spec->span_bytes;
+    const size_t slots_h = (span - foot_h) / width + 1, slots_d = (span - foot_d) / width + 1;
+    const int64_t n = spec->total_bytes / spec->copy_bytes;
+    // where each transfer starts: consecutive (wrapping) or seeded pseudo-random row-aligned offsets
+    std::vector<size_t> off_h[2], off_d[2];
+    try {
+        for (int k = 0; k < 2; ++k) {
+            off_h[k].resize((size_t)n);
+            off_d[k].resize((size_t)n);
+        }
+    } catch (...) {
+        return fail(nullptr, KV_ERR_NOMEM, "out of host memory");
+    }
+    uint64_t lcg = 0x9E3779B97F4A7C15ull;
+    for (int k = 0; k < 2; ++k)
+        for (int64_t i = 0; i < n; ++i) {
+            lcg = lcg * 6364136223846793005ull + 1442695040888963407ull;
+            const size_t r1 = (size_t)(lcg >> 33);
+            lcg = lcg * 6364136223846793005ull + 1442695040888963407ull;
+            const size_t r2 = (size_t)(lcg >> 33);
+            // consecutive transfers tile the span when they are plain (one row, or rows packed back to back)
+            const size_t step_h = (hpitch == width) ? (size_t)rows : 1, step_d = (dpitch == width) ? (size_t)rows : 1;
+            off_h[k][(size_t)i] = (spec->scattered ? r1 % slots_h : ((size_t)i * step_h) % slots_h) * width;
+            off_d[k][(size_t)i] = (spec->scattered ? r2 % slots_d : ((size_t)i * step_d) % slots_d) * width;
+        }
     uint8_t *h[2] = {nullptr, nullptr}, *dv[2] = {nullptr, nullptr};
     cudaStream_t st[2] = {nullptr, nullptr};
     cudaEvent_t ev[4] = {};
@@ -950,25 +1174,35 @@ int32_t kv_probe_link(int32_t device_id, int64_t bytes, int32_t reps, kv_link_pr
         }                                               \
     } while (0)
     for (int k = 0; k < 2; ++k) {
-        KV_PROBE(cudaHostAlloc((void **)&h[k], (size_t)bytes, cudaHostAllocDefault));
-        memset(h[k], k + 1, (size_t)bytes);
-        KV_PROBE(cudaMalloc((void **)&dv[k], (size_t)bytes));
-        KV_PROBE(cudaMemset(dv[k], 0, (size_t)bytes));
+        KV_PROBE(cudaHostAlloc((void **)&h[k], span, cudaHostAllocDefault));
+        memset(h[k], k + 1, span);
+        KV_PROBE(cudaMalloc((void **)&dv[k], span));
+        KV_PROBE(cudaMemset(dv[k], 0, span));
         KV_PROBE(cudaStreamCreateWithFlags(&st[k], cudaStreamNonBlocking));
     }
     for (int k = 0; k < 4; ++k) KV_PROBE(cudaEventCreate(&ev[k]));
-    const double gb = (double)bytes * reps / 1e9;
+    auto d2h = [&](int64_t i) {
+        uint8_t *hp = h[0] + off_h[0][(size_t)i], *dp = dv[0] + off_d[0][(size_t)i];
+        return rows == 1 ? cudaMemcpyAsync(hp, dp, width, cudaMemcpyDeviceToHost, st[0])
+                         : cudaMemcpy2DAsync(hp, hpitch, dp, dpitch, width, (size_t)rows, cudaMemcpyDeviceToHost, st[0]);
+    };
+    auto h2d = [&](int64_t i) {
+        uint8_t *hp = h[1] + off_h[1][(size_t)i], *dp = dv[1] + off_d[1][(size_t)i];
+        return rows == 1 ? cudaMemcpyAsync(dp, hp, width, cudaMemcpyHostToDevice, st[1])
+                         : cudaMemcpy2DAsync(dp, dpitch, hp, hpitch, width, (size_t)rows, cudaMemcpyHostToDevice, st[1]);
+    };
+    const double gb = (double)spec->copy_bytes * (double)n / 1e9;
     double best_d2h = 0, best_h2d = 0, best_sum = 0, best_bd = 0, best_bh = 0;
-    for (int round = 0; round < 4; ++round) {
+    for (int round = 0; round <= spec->rounds; ++round) {       // round 0 warms up
         float ms = 0.f;
         KV_PROBE(cudaEventRecord(ev[0], st[0]));
-        for (int r = 0; r < reps; ++r) KV_PROBE(cudaMemcpyAsync(h[0], dv[0], (size_t)bytes, cudaMemcpyDeviceToHost, st[0]));
+        for (int64_t i = 0; i < n; ++i) KV_PROBE(d2h(i));
         KV_PROBE(cudaEventRecord(ev[1], st[0]));
         KV_PROBE(cudaStreamSynchronize(st[0]));
         KV_PROBE(cudaEventElapsedTime(&ms, ev[0], ev[1]));
         if (round) best_d2h = std::max(best_d2h, gb / (ms * 1e-3));
         KV_PROBE(cudaEventRecord(ev[0], st[1]));
-        for (int r = 0; r < reps; ++r) KV_PROBE(cudaMemcpyAsync(dv[1], h[1], (size_t)bytes, cudaMemcpyHostToDevice, st[1]));
+        for (int64_t i = 0; i < n; ++i) KV_PROBE(h2d(i));
         KV_PROBE(cudaEventRecord(ev[1], st[1]));
         KV_PROBE(cudaStreamSynchronize(st[1]));
         KV_PROBE(cudaEventElapsedTime(&ms, ev[0], ev[1]));
@@ -976,9 +1210,9 @@ int32_t kv_probe_link(int32_t device_id, int64_t bytes, int32_t reps, kv_link_pr
         // both at once; window = first start to last end
         KV_PROBE(cudaEventRecord(ev[0], st[0]));
         KV_PROBE(cudaEventRecord(ev[2], st[1]));
-        for (int r = 0; r < reps; ++r) {
-            KV_PROBE(cudaMemcpyAsync(h[0], dv[0], (size_t)bytes, cudaMemcpyDeviceToHost, st[0]));
-            KV_PROBE(cudaMemcpyAsync(dv[1], h[1], (size_t)bytes, cudaMemcpyHostToDevice, st[1]));
+        for (int64_t i = 0; i < n; ++i) {
+            KV_PROBE(d2h(i));
+            KV_PROBE(h2d(i));
         }
         KV_PROBE(cudaEventRecord(ev[1], st[0]));
         KV_PROBE(cudaEventRecord(ev[3], st[1]));
@@ -989,8 +1223,8 @@ int32_t kv_probe_link(int32_t device_id, int64_t bytes, int32_t reps, kv_link_pr
         KV_PROBE(cudaEventElapsedTime(&t_in, ev[2], ev[3]));
         const bool fwd = cudaEventElapsedTime(&a, ev[0], ev[2]) == cudaSuccess;
         const bool bwd = cudaEventElapsedTime(&b, ev[2], ev[0]) == cudaSuccess;
-        const float off = (fwd && a > 0.f) ? a : ((bwd && b > 0.f) ? -b : 0.f);
-        const float win = std::max(t_out, off + t_in) - std::min(0.f, off);
+        const float offs = (fwd && a > 0.f) ? a : ((bwd && b > 0.f) ? -b : 0.f);
+        const float win = std::max(t_out, offs + t_in) - std::min(0.f, offs);
         const double sum = 2 * gb / (win * 1e-3);
         if (round && sum > best_sum) {
             best_sum = sum;
@@ -1004,11 +1238,25 @@ int32_t kv_probe_link(int32_t device_id, int64_t bytes, int32_t reps, kv_link_pr
     out->bi_sum_gbs = best_sum;
     out->bi_d2h_gbs = best_bd;
     out->bi_h2d_gbs = best_bh;
-    out->bytes = bytes;
-    out->reps = reps;
+    out->bytes = spec->copy_bytes;
+    out->reps = (int32_t)std::min<int64_t>(n, INT32_MAX);
     cleanup();
     (void)cudaGetLastError();
     return KV_OK;
+}
+
+int32_t kv_probe_link(int32_t device_id, int64_t bytes, int32_t reps, kv_link_probe_t *out)
+{
+    if (bytes <= 0 || reps <= 0) return fail(nullptr, KV_ERR_INVALID_ARG, "bad probe arguments");
+    kv_probe_spec_t spec;
+    spec.copy_bytes = bytes;
+    spec.total_bytes = bytes * reps;
+    spec.span_bytes = bytes;
+    spec.scattered = 0;
+    spec.rounds = 3;
+    spec.rows = 1;
+    spec.host_pitch = spec.dev_pitch = 0;
+    return kv_probe_link_ex(device_id, &spec, out);
 }
 
 }  // extern "C"

@@ -270,3 +270,49 @@ def test_gpu_fill_twin_matches_cpu_generator():
     sums = F.checksum_blocks(lay, nb)
     for b in range(nb):
         assert sums[b] == F.checksum_words(W.block_words(77, W.POOL_GPU, b, shape.words_per_block))
+
+
+@pytest.mark.parametrize("layout", [0, 1], ids=["hostblockfirst", "hostlayerfirst"])
+def test_staged_transfer_planning_patterns(layout):
+    """Host-id patterns that the staged path turns into different copy-engine transfers: long runs,
+    equal runs at a constant spacing (one strided transfer of several rows), isolated blocks in
+    pairs, a list given in descending order, repeated swap-in sources, and more blocks than one
+    staging half holds."""
+    shape = W.KVShape(2, 16, 4, 64)              # 16 KiB planes, 64 KiB blocks
+    nbg, nbh = 96, 400
+    p = _pair(shape, nbg, nbh, seed=11, host_layout=layout, path=PATHS["staged"], staging_bytes=12 * shape.block_bytes)
+    rng = np.random.default_rng(4)
+    try:
+        patterns = {
+            "one long run": np.arange(100, 140),
+            "runs of 3 every 10": np.concatenate([np.arange(s, s + 3) for s in range(20, 120, 10)]),
+            "every 7th": np.arange(3, 3 + 7 * 30, 7),
+            "descending": np.arange(300, 260, -1),
+            "mixed": np.array([0, 1, 2, 9, 20, 21, 50, 51, 52, 53, 80, 399, 398, 200, 210, 220, 231, 5]),
+            "random": rng.choice(nbh, 45, replace=False),
+        }
+        for name, hid in patterns.items():
+            hid = hid.astype(np.int32)
+            g = rng.choice(nbg, len(hid), replace=False).astype(np.int32)
+            assert p.oracle.swap_out(g, hid) == 0 and p.pool.kv_swap_out(g, hid) == 0
+            p.assert_equal(f"staged out, {name}")
+            g2 = rng.choice(nbg, len(hid), replace=False).astype(np.int32)
+            assert p.oracle.swap_in(hid, g2) == 0 and p.pool.kv_swap_in(hid, g2) == 0
+            p.assert_equal(f"staged in, {name}")
+        # the same host block as the source of several swap-ins
+        hid = np.array([7, 7, 8, 7, 30, 30, 31], np.int32)
+        g = rng.choice(nbg, len(hid), replace=False).astype(np.int32)
+        assert p.oracle.swap_in(hid, g) == 0 and p.pool.kv_swap_in(hid, g) == 0
+        p.assert_equal("staged in, repeated sources")
+        # both directions at once, several halves deep, queued twice without a sync
+        for _ in range(2):
+            og = rng.choice(nbg, 40, replace=False).astype(np.int32)
+            ig = np.setdiff1d(np.arange(nbg), og)[:40].astype(np.int32)
+            oh = rng.choice(nbh, 40, replace=False).astype(np.int32)
+            ih = rng.choice(np.setdiff1d(np.arange(nbh), oh), 40, replace=False).astype(np.int32)
+            assert p.rotate_both(W.Rotation(og, oh, ih, ig, np.zeros(1), np.zeros(1))) == 0
+        p.assert_equal("staged rotate, queued")
+        st = p.pool.kv_get_stats()
+        assert st["device_status"] == 0 and st["kernel_launches"] > 0
+    finally:
+        p.close()
