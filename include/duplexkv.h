@@ -204,7 +204,7 @@ int32_t kv_probe_link(int32_t device_id, int64_t bytes, int32_t reps, kv_link_pr
 
 /*
  * The same probe with the shape of the transfers as parameters: the bandwidth-versus-transfer-size
- * curve of the paper's motivation study (the figure of section 3.2 on full-duplex bandwidth against
+ * curve of the paper's motivation study (the figure of section 3.3 on full-duplex bandwidth against
  * segment size, and the launch-versus-transfer-time figure of section 4.3.1).  Each round issues
  * total_bytes/copy_bytes copy-engine transfers of copy_bytes back to back on one stream per direction.
  * rows <= 1: plain transfers.  rows > 1: strided 2-D transfers of `rows` rows of copy_bytes/rows bytes,

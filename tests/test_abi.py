@@ -1,0 +1,48 @@
+"""The C-ABI library loads without a GPU and exports every function ``include/duplexkv.h`` declares;
+the Python binding names the same set.  No compute call is made here."""
+import ctypes as C
+import os
+import re
+
+from paper_2601_20309_b200 import binding as B
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+def declared_functions():
+    text = open(os.path.join(ROOT, "include", "duplexkv.h")).read()
+    text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)                   # drop comments
+    return sorted(set(re.findall(r"^\s*(?:const\s+char\s*\*|int32_t|int64_t)\s*(kv_[a-z0-9_]+)\s*\(", text, flags=re.M)))
+
+
+def test_header_declares_the_named_calls():
+    names = declared_functions()
+    for must in ("kv_pool_create", "kv_swap_out", "kv_swap_in", "kv_rotate", "kv_sync"):
+        assert must in names
+    assert len(names) >= 15
+
+
+def test_library_exports_every_declared_symbol():
+    lib = B.lib()
+    missing = [n for n in declared_functions() if not hasattr(lib, n)]
+    assert not missing, missing
+
+
+def test_binding_names_match_the_header():
+    assert sorted(B.EXPORTS) == declared_functions()
+
+
+def test_shape_helpers_need_no_device():
+    assert B.kv_seg_bytes(16, 8, 128) == 32768
+    assert B.kv_blk_bytes(32, 16, 8, 128) == 2 << 20
+    assert B.kv_blk_bytes(80, 16, 8, 128) == 5 << 20
+    assert B.kv_seg_bytes(0, 8, 128) == 0
+    assert B.kv_path_for(2 << 20) == B.KV_PATH_STAGED and B.kv_path_for(1 << 20) == B.KV_PATH_ZEROCOPY
+
+
+def test_struct_sizes_match_the_header_layout():
+    # natural alignment on both sides; a mismatch here means the ctypes mirror drifted from the header
+    assert C.sizeof(B.kv_pool_config_t) == 104
+    assert C.sizeof(B.kv_stats_t) == 112
+    assert C.sizeof(B.kv_link_probe_t) == 56
+    assert C.sizeof(B.kv_probe_spec_t) == 56
