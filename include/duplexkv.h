@@ -178,6 +178,42 @@ int32_t kv_sync(kv_pool_t *pool);
 int32_t kv_gather_blocks(kv_pool_t *pool, const int32_t *gpu_ids, int64_t n, void *dst_device);
 int32_t kv_scatter_blocks(kv_pool_t *pool, const void *src_device, const int32_t *gpu_ids, int64_t n);
 
+/*
+ * kv_gather_blocks for callers that cannot allocate.  (The paper has no counterpart: its engine
+ * allocates freely.  This exists for users of this library.)
+ *
+ * Who that is: code that runs where a cudaMalloc is off limits -- inside a serving loop that must
+ * not take the device-wide synchronisation an allocation or a free implies, in a process whose
+ * whole GPU memory already belongs to another allocator, or in a component that is handed its
+ * buffers and may not create any.  A pool (kv_pool_create) allocates descriptor rings, events and
+ * staging, so such callers cannot hold one; this entry point needs none.
+ *
+ * Same result as kv_gather_blocks: the listed blocks of the layer-first pool at device_base
+ * (num_gpu_blocks blocks of the given shape) are written, in list order, to dst_device block-first
+ * (block i at i*BLK, planes in (layer, K|V) order).  device_base, dst_device: DEVICE pointers on the
+ * CURRENT device, 16-byte aligned, dst_device holding n*BLK bytes.  gpu_ids: HOST pointer, ids may
+ * repeat.  stream: a cudaStream_t of the current device, or NULL for the default stream.
+ *
+ * The id list the kernel walks and the kernel's status word sit in an array built into the library
+ * (KV_STATIC_MAX_BLOCKS ids, 64.25 KiB of device memory on every GPU that loads the library, held
+ * until the process exits).  n > KV_STATIC_MAX_BLOCKS is refused with KV_ERR_INVALID_ARG and a
+ * message in kv_last_error(NULL); split longer lists.  The call makes no cudaMalloc, cudaFree,
+ * cudaHostAlloc or stream / event creation.  It is SYNCHRONOUS: it returns when the gather has
+ * finished (KV_OK), or with KV_ERR_RANGE / KV_ERR_INVALID_ARG / KV_ERR_UNSUPPORTED before anything
+ * ran, or KV_ERR_CUDA / KV_ERR_TIMEOUT.
+ *
+ * The first call on each device looks up the array's device address and sets the kernel's
+ * shared-memory limit for that device; make that first call before starting any stream capture.
+ * All calls share the one array, which still holds the previous call's ids (they are overwritten,
+ * and the status word is cleared, at the start of each call): two calls that overlap in time -- from
+ * two threads, or on two streams -- race on it, also across different pools or shapes.  One call at
+ * a time per device.
+ */
+#define KV_STATIC_MAX_BLOCKS 8192
+int32_t kv_gather_blocks_static(const void *device_base, int32_t num_layers, int32_t block_size,
+                                int32_t kv_heads, int32_t head_dim, int64_t num_gpu_blocks,
+                                const int32_t *gpu_ids, int64_t n, void *dst_device, void *stream);
+
 /* Host pool base (HOST pointer) and size, for filling and verification. */
 int32_t kv_host_ptr(kv_pool_t *pool, void **base, int64_t *bytes);
 

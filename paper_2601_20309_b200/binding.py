@@ -72,7 +72,8 @@ class kv_probe_spec_t(C.Structure):
 
 EXPORTS = ["kv_pool_create", "kv_pool_destroy", "kv_pool_set_path", "kv_swap_out", "kv_swap_in", "kv_rotate", "kv_sync",
            "kv_gather_blocks", "kv_scatter_blocks", "kv_host_ptr", "kv_get_stats", "kv_last_error",
-           "kv_seg_bytes", "kv_blk_bytes", "kv_path_for", "kv_probe_link", "kv_probe_link_ex"]
+           "kv_seg_bytes", "kv_blk_bytes", "kv_path_for", "kv_probe_link", "kv_probe_link_ex",
+           "kv_gather_blocks_static"]
 
 _lib = None
 
@@ -117,6 +118,8 @@ def lib() -> C.CDLL:
     L.kv_path_for.argtypes = [i64]
     L.kv_probe_link.restype = C.c_int32
     L.kv_probe_link.argtypes = [C.c_int32, i64, C.c_int32, C.POINTER(kv_link_probe_t)]
+    L.kv_gather_blocks_static.restype = C.c_int32
+    L.kv_gather_blocks_static.argtypes = [vp, C.c_int32, C.c_int32, C.c_int32, C.c_int32, i64, i32p, i64, vp, vp]
     L.kv_probe_link_ex.restype = C.c_int32
     L.kv_probe_link_ex.argtypes = [C.c_int32, C.POINTER(kv_probe_spec_t), C.POINTER(kv_link_probe_t)]
     _lib = L
@@ -167,6 +170,22 @@ def kv_probe_link_ex(device_id: int, copy_bytes: int, total_bytes: int, span_byt
     if rc != KV_OK:
         raise KVError(rc, lib().kv_last_error(None).decode())
     return {k: getattr(out, k) for k, _ in kv_link_probe_t._fields_ if k != "pad_"}
+
+
+KV_STATIC_MAX_BLOCKS = 8192
+
+
+def kv_gather_blocks_static(device_base: int, num_layers: int, block_size: int, kv_heads: int, head_dim: int,
+                            num_gpu_blocks: int, gpu_ids, dst_device: int, stream: Optional[int] = None,
+                            check: bool = True) -> int:
+    """The allocation-free gather (no pool needed): see ``kv_gather_blocks_static`` in the header.
+    Synchronous; one call at a time per device."""
+    g, gp = _ids(gpu_ids)
+    rc = lib().kv_gather_blocks_static(device_base, num_layers, block_size, kv_heads, head_dim, num_gpu_blocks,
+                                       gp, len(g), dst_device, stream)
+    if check and rc != KV_OK:
+        raise KVError(rc, lib().kv_last_error(None).decode())
+    return rc
 
 
 class KVPool:

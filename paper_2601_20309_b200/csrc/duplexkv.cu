@@ -1260,3 +1260,93 @@ int32_t kv_probe_link(int32_t device_id, int64_t bytes, int32_t reps, kv_link_pr
 }
 
 }  // extern "C"
+
+// =================================================================================================
+// Gather without any allocation.
+//
+// Some programs that want the gather cannot allocate CUDA memory at the point where they call it:
+// a serving loop that must not hit the device-wide synchronisation cudaMalloc / cudaFree imply, a
+// process whose device memory is entirely owned by another allocator (a framework's caching pool
+// that was sized to the whole GPU), or a plug-in that is handed buffers and forbidden to make its
+// own.  kv_pool_create allocates (descriptor rings, events, staging), so those callers cannot use
+// a pool.  For them the id list that the copy kernel walks, and the status word its bounded waits
+// report to, live in this fixed array, which every GPU that loads the library carries until exit.
+#define KV_STATIC_STATUS_WORDS 64      // 256 bytes after the pairs; word 0 is the status word
+static __device__ __align__(256) int2 kv_static_scratch[KV_STATIC_MAX_BLOCKS + KV_STATIC_STATUS_WORDS / 2];
+
+namespace {
+constexpr int KV_MAX_DEVICES = 64;
+// device address of kv_static_scratch per device ordinal (in host code the array's name is only a
+// host-side handle; kernels must be given the address cudaGetSymbolAddress returns)
+void *g_static_scratch[KV_MAX_DEVICES] = {};
+int2 g_static_pairs_host[KV_STATIC_MAX_BLOCKS];
+}  // namespace
+
+extern "C" int32_t kv_gather_blocks_static(const void *device_base, int32_t num_layers, int32_t block_size,
+                                           int32_t kv_heads, int32_t head_dim, int64_t num_gpu_blocks,
+                                           const int32_t *gpu_ids, int64_t n, void *dst_device, void *stream)
+{
+    const int64_t seg = kv_seg_bytes(block_size, kv_heads, head_dim);
+    const int64_t blk = kv_blk_bytes(num_layers, block_size, kv_heads, head_dim);
+    if (seg <= 0 || blk <= 0 || num_gpu_blocks <= 0 || num_gpu_blocks > INT32_MAX || seg > (1 << 30) ||
+        2 * (int64_t)num_layers > (1 << 20))
+        return fail(nullptr, KV_ERR_INVALID_ARG, "bad shape or pool size");
+    if (seg % 16 != 0) return fail(nullptr, KV_ERR_UNSUPPORTED, "segment size must be a multiple of 16 bytes");
+    if (n < 0) return fail(nullptr, KV_ERR_INVALID_ARG, "negative count");
+    if (n == 0) return KV_OK;
+    if (n > KV_STATIC_MAX_BLOCKS) {
+        snprintf(g_err, 256, "n = %lld exceeds KV_STATIC_MAX_BLOCKS = %d, the capacity of the built-in id scratch",
+                 (long long)n, KV_STATIC_MAX_BLOCKS);
+        return KV_ERR_INVALID_ARG;
+    }
+    if (!device_base || !gpu_ids || !dst_device) return fail(nullptr, KV_ERR_INVALID_ARG, "null argument");
+    if (((uintptr_t)device_base & 15) || ((uintptr_t)dst_device & 15))
+        return fail(nullptr, KV_ERR_INVALID_ARG, "device_base and dst_device must be 16-byte aligned");
+    for (int64_t i = 0; i < n; ++i) {
+        if (gpu_ids[i] < 0 || (int64_t)gpu_ids[i] >= num_gpu_blocks) {
+            snprintf(g_err, 256, "gpu_ids[%lld] = %d outside [0, %lld)", (long long)i, gpu_ids[i], (long long)num_gpu_blocks);
+            return KV_ERR_RANGE;
+        }
+        g_static_pairs_host[i] = make_int2(gpu_ids[i], (int)i);
+    }
+    int dev = -1;
+    KV_CUDA(nullptr, cudaGetDevice(&dev));
+    if (dev < 0 || dev >= KV_MAX_DEVICES) return fail(nullptr, KV_ERR_UNSUPPORTED, "device ordinal beyond the table");
+    if (!g_static_scratch[dev]) {
+        // once per device, with that device current
+        void *ptr = nullptr;
+        KV_CUDA(nullptr, cudaGetSymbolAddress((void **)&ptr, kv_static_scratch));
+        KV_CUDA(nullptr, cudaFuncSetAttribute(kv_copy_bulk<BULK_STAGE, BULK_NS, BULK_AHEAD>,
+                                              cudaFuncAttributeMaxDynamicSharedMemorySize, BULK_STAGE * BULK_NS));
+        g_static_scratch[dev] = ptr;
+    }
+    int2 *pairs = (int2 *)g_static_scratch[dev];
+    unsigned int *status = (unsigned int *)(pairs + KV_STATIC_MAX_BLOCKS);
+    cudaStream_t st = (cudaStream_t)stream;
+    int sm_count = 0;
+    KV_CUDA(nullptr, cudaDeviceGetAttribute(&sm_count, cudaDevAttrMultiProcessorCount, dev));
+
+    // the array keeps the previous call's contents: the pairs are overwritten, the status word is cleared
+    KV_CUDA(nullptr, cudaMemcpyAsync(pairs, g_static_pairs_host, (size_t)n * sizeof(int2), cudaMemcpyHostToDevice, st));
+    KV_CUDA(nullptr, cudaMemsetAsync(status, 0, sizeof(unsigned int), st));
+    KvJob job;
+    job.planes = 2 * num_layers;
+    job.seg = (int)seg;
+    job.chunk = (int)std::min<int64_t>(seg, BULK_STAGE);
+    job.cps = (int)((seg + job.chunk - 1) / job.chunk);
+    job.status = status;
+    job.dir[1] = KvDir{};
+    KvDir &kd = job.dir[0];
+    kd.src = KvSide{(unsigned long long)device_base, seg, num_gpu_blocks * seg};
+    kd.dst = KvSide{(unsigned long long)dst_device, blk, seg};
+    kd.pairs = pairs;
+    kd.n = (int)n;
+    kd.ctas = clamp_ctas(job, kd, sm_count > 0 ? sm_count : 1);
+    kv_copy_bulk<BULK_STAGE, BULK_NS, BULK_AHEAD><<<kd.ctas, 32, BULK_STAGE * BULK_NS, st>>>(job);
+    KV_CUDA(nullptr, cudaGetLastError());
+    unsigned int seen = 0;
+    KV_CUDA(nullptr, cudaMemcpyAsync(&seen, status, sizeof(seen), cudaMemcpyDeviceToHost, st));
+    KV_CUDA(nullptr, cudaStreamSynchronize(st));
+    if (seen & KV_DEV_TIMEOUT) return fail(nullptr, KV_ERR_TIMEOUT, "a device-side wait ran out");
+    return KV_OK;
+}
