@@ -1,0 +1,145 @@
+"""Measurement sweeps on the GPU machine (need a CUDA device).
+
+    python -m paper_2601_20309_b200.sweep probe [--out FILE]
+        The host link's bandwidth against the shape of copy-engine transfers: plain transfers of
+        32 KiB .. 1 GiB, and strided 2-D transfers (rows x row bytes), each direction alone and both
+        at once, at scattered offsets of 4 GiB pinned buffers.  The analogue of the paper's
+        bandwidth-versus-segment-size figure (section 3.3) on this machine.
+
+    python -m paper_2601_20309_b200.sweep paths [--max-payload-gb G] [--out FILE]
+        Block-size and fragmentation sweep on the 8B shape: block_size 8/16/32/64, block tables
+        contiguous or uniformly random, payload 64 MB .. G GB per direction, each direction alone
+        and both at once, on every transfer path.  Its result is the table behind kv_path_for.
+
+Both print one JSON object per line and, at the end, a markdown table.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import sys
+
+from . import binding as B
+from . import workload as W
+
+K, M, G = 1 << 10, 1 << 20, 1 << 30
+
+
+def _emit(rec, out):
+    line = json.dumps(rec)
+    print(line, flush=True)
+    if out:
+        out.write(line + "\n")
+        out.flush()
+
+
+def probe(out) -> None:
+    rows = []
+    base = B.kv_probe_link(0, 256 * M, 4)
+    _emit({"case": "reference: 256 MiB plain transfers, same buffer", **base}, out)
+    shapes = [(f"plain {s // K} KiB" if s < M else f"plain {s // M} MiB", dict(copy_bytes=s))
+              for s in (32 * K, 64 * K, 256 * K, 1 * M, 2 * M, 4 * M, 8 * M, 16 * M, 64 * M, 256 * M, 1 * G)]
+    shapes += [
+        ("64 rows x 32 KiB, packed both sides", dict(copy_bytes=2 * M, rows=64)),
+        ("64 rows x 32 KiB, device pitch 32 MiB (one block-16 block of a layer-first pool)",
+         dict(copy_bytes=2 * M, rows=64, dev_pitch=32 * M)),
+        ("64 rows x 16 KiB, device pitch 32 MiB (block 8)", dict(copy_bytes=1 * M, rows=64, dev_pitch=32 * M)),
+        ("64 rows x 64 KiB, device pitch 32 MiB (block 32)", dict(copy_bytes=4 * M, rows=64, dev_pitch=32 * M)),
+        ("64 rows x 128 KiB, device pitch 32 MiB (block 64)", dict(copy_bytes=8 * M, rows=64, dev_pitch=32 * M)),
+        ("2 rows x 1 MiB, host pitch 64 MiB", dict(copy_bytes=2 * M, rows=2, host_pitch=64 * M)),
+        ("2 rows x 2 MiB, host pitch 64 MiB", dict(copy_bytes=4 * M, rows=2, host_pitch=64 * M)),
+        ("2 rows x 2 MiB, host pitch 1 GiB", dict(copy_bytes=4 * M, rows=2, host_pitch=1024 * M)),
+        ("2 rows x 4 MiB, host pitch 64 MiB", dict(copy_bytes=8 * M, rows=2, host_pitch=64 * M)),
+        ("4 rows x 2 MiB, host pitch 64 MiB", dict(copy_bytes=8 * M, rows=4, host_pitch=64 * M)),
+        ("8 rows x 2 MiB, host pitch 64 MiB", dict(copy_bytes=16 * M, rows=8, host_pitch=64 * M)),
+    ]
+    for name, kw in shapes:
+        total = G if kw["copy_bytes"] >= 256 * K else G // 4
+        r = B.kv_probe_link_ex(0, total_bytes=max(total, kw["copy_bytes"]), span_bytes=4 * G, scattered=True,
+                               rounds=2, **kw)
+        rec = {"case": name, **{k: round(v, 2) for k, v in r.items() if k.endswith("gbs")},
+               "transfers_per_round": r["reps"]}
+        rows.append(rec)
+        _emit(rec, out)
+    print("\n| transfer shape | D2H alone | H2D alone | both: D2H | both: H2D | both: sum |\n|---|---|---|---|---|---|")
+    for r in rows:
+        print(f"| {r['case']} | {r['d2h_gbs']} | {r['h2d_gbs']} | {r['bi_d2h_gbs']} | {r['bi_h2d_gbs']} | {r['bi_sum_gbs']} |")
+
+
+PATHS = [("staged", B.KV_PATH_STAGED), ("zerocopy", B.KV_PATH_ZEROCOPY), ("ce2d", B.KV_PATH_CE2D),
+         ("naive", B.KV_PATH_NAIVE)]
+
+
+def paths(out, max_payload_gb: float) -> None:
+    import torch
+    rows = []
+    payloads = [p for p in (64e6, 256e6, 1e9, 4e9, 8e9) if p <= max_payload_gb * 1e9 + 1]
+    for bs in (8, 16, 32, 64):
+        for contiguous in (True, False):
+            for payload in payloads:
+                shape = W.KVShape(32, bs)
+                n = max(1, int(payload // shape.block_bytes))
+                # random tables: a host pool much larger than the payload, so that ids are truly scattered
+                nb_host = 2 * n + 16 if contiguous else int(min(16 * n, 40e9 // shape.block_bytes))
+                w = W.config4_sweep_case(bs, contiguous, payload, nb_host=max(nb_host, 2 * n + 16))
+                rot = w.steps[0]
+                dev = torch.empty(w.nb_gpu * shape.block_bytes, dtype=torch.uint8, device="cuda:0")
+                probe_bi = B.kv_probe_link(0, 256 * M, 2)["bi_sum_gbs"]
+                pool = B.KVPool(shape.num_layers, shape.block_size, shape.kv_heads, shape.head_dim, w.nb_gpu,
+                                w.nb_host, dev.data_ptr())
+                nbytes = rot.n_out * shape.block_bytes
+
+                def best(fn, reps):
+                    ts = []
+                    for k in range(reps + 1):
+                        fn()
+                        pool.kv_sync()
+                        if k:
+                            ts.append(pool.kv_get_stats()["last_union_ms"])
+                    return min(ts)
+
+                rec = {"block_size": bs, "seg_kib": shape.words_per_plane * 2 // K, "blk_mib": shape.block_bytes / M,
+                       "tables": "contiguous" if contiguous else "random", "payload_mb": round(nbytes / 1e6),
+                       "blocks": rot.n_out, "probe_bi_gbs": round(probe_bi, 1)}
+                for name, pid in PATHS:
+                    if name == "naive" and payload > 300e6:
+                        continue
+                    pool.kv_pool_set_path(pid, pid)
+                    reps = 1 if name == "naive" else 3
+                    t_o = best(lambda: pool.kv_swap_out(rot.out_gpu, rot.out_host), reps)
+                    t_i = best(lambda: pool.kv_swap_in(rot.in_host, rot.in_gpu), reps)
+                    t_b = best(lambda: pool.kv_rotate(rot.out_gpu, rot.out_host, rot.in_host, rot.in_gpu), reps)
+                    rec[name] = {"out": round(nbytes / t_o / 1e6, 1), "in": round(nbytes / t_i / 1e6, 1),
+                                 "both": round(2 * nbytes / t_b / 1e6, 1)}
+                pool.destroy()
+                del dev
+                torch.cuda.empty_cache()
+                rec["auto"] = B.PATH_NAMES[B.kv_path_for(shape.block_bytes)]
+                rows.append(rec)
+                _emit(rec, out)
+    print("\n| block | BLK MiB | tables | payload MB | probe both | staged out/in/both | zero-copy out/in/both | "
+          "2-D per block out/in/both | per segment out/in/both | AUTO |\n|---|---|---|---|---|---|---|---|---|---|")
+    for r in rows:
+        f = lambda k: "%s / %s / %s" % (r[k]["out"], r[k]["in"], r[k]["both"]) if k in r else "-"
+        print(f"| {r['block_size']} | {r['blk_mib']:g} | {r['tables']} | {r['payload_mb']} | {r['probe_bi_gbs']} | "
+              f"{f('staged')} | {f('zerocopy')} | {f('ce2d')} | {f('naive')} | {r['auto']} |")
+
+
+def main() -> None:
+    ap = argparse.ArgumentParser()
+    ap.add_argument("what", choices=["probe", "paths"])
+    ap.add_argument("--out", default=None)
+    ap.add_argument("--max-payload-gb", type=float, default=4.0)
+    a = ap.parse_args()
+    import torch
+    if not torch.cuda.is_available():
+        sys.exit("sweep needs a CUDA device")
+    out = open(a.out, "w") if a.out else None
+    if a.what == "probe":
+        probe(out)
+    else:
+        paths(out, a.max_payload_gb)
+
+
+if __name__ == "__main__":
+    main()
