@@ -384,7 +384,8 @@ int32_t plan_staged(kv_pool *p, DirCall &c)
     return KV_OK;
 }
 
-int32_t begin_dir(kv_pool *p, DirCall &c, bool wait_other)
+// wait_for: end event of the other direction's call this one must follow, or nullptr
+int32_t begin_dir(kv_pool *p, DirCall &c, cudaEvent_t wait_for)
 {
     DirState &s = p->dir[c.d];
     const uint64_t seq = s.issued + 1;
@@ -415,10 +416,7 @@ int32_t begin_dir(kv_pool *p, DirCall &c, bool wait_other)
         for (int64_t i = 0; i < c.n; ++i)
             c.pairs_host[i] = (c.d == 0) ? make_int2(c.gpu_ids[i], c.host_ids[i]) : make_int2(c.host_ids[i], c.gpu_ids[i]);
     }
-    if (wait_other) {
-        DirState &o = p->dir[1 - c.d];
-        KV_CUDA(p, cudaStreamWaitEvent(s.stream, o.ev_end[o.issued % KV_SLOTS], 0));
-    }
+    if (wait_for) KV_CUDA(p, cudaStreamWaitEvent(s.stream, wait_for, 0));
     KV_CUDA(p, cudaEventRecord(s.ev_start[c.slot], s.stream));
     if (c.path == KV_PATH_ZEROCOPY) {
         KV_CUDA(p, cudaMemcpyAsync(c.pairs_dev, c.pairs_host, (size_t)c.n * sizeof(int2), cudaMemcpyHostToDevice, s.stream));
@@ -625,6 +623,16 @@ int32_t issue_calls(kv_pool *p, DirCall *calls, int ncalls, bool fused)
 int32_t run_calls(kv_pool *p, DirCall *calls, int ncalls, const bool *wait_other, bool fused)
 {
     p->union_slot[0] = p->union_slot[1] = -1;
+    // The event each call has to wait for is the end of the other direction's latest EARLIER call.  It is
+    // looked up here, before any direction of this call is begun: beginning the swap-out advances that
+    // direction's call counter, and the swap-in of the same rotate must not mistake the swap-out it
+    // travels with (whose end event is not recorded yet) for the earlier call it depends on.
+    cudaEvent_t wait_ev[2] = {nullptr, nullptr};
+    for (int k = 0; k < ncalls; ++k)
+        if (wait_other[k]) {
+            const DirState &o = p->dir[1 - calls[k].d];
+            wait_ev[k] = o.ev_end[o.issued % KV_SLOTS];
+        }
     for (int k = 0; k < ncalls; ++k) {
         calls[k].path = resolve_path(p, calls[k].d);
         if (fused && calls[k].d == 1) {
@@ -639,7 +647,7 @@ int32_t run_calls(kv_pool *p, DirCall *calls, int ncalls, const bool *wait_other
         cudaStream_t keep = p->dir[1].stream;
         p->dir[1].stream = p->dir[0].stream;
         int32_t rc = KV_OK;
-        for (int k = 0; k < ncalls && rc == KV_OK; ++k) rc = begin_dir(p, calls[k], wait_other[k]);
+        for (int k = 0; k < ncalls && rc == KV_OK; ++k) rc = begin_dir(p, calls[k], wait_ev[k]);
         if (rc == KV_OK) rc = issue_calls(p, calls, ncalls, true);
         for (int k = 0; k < ncalls && rc == KV_OK; ++k) rc = end_dir(p, calls[k]);
         p->dir[1].stream = keep;
@@ -647,7 +655,7 @@ int32_t run_calls(kv_pool *p, DirCall *calls, int ncalls, const bool *wait_other
         KV_CUDA(p, cudaStreamWaitEvent(keep, p->dir[1].ev_end[calls[1].slot], 0));
     } else {
         for (int k = 0; k < ncalls; ++k) {
-            int32_t rc = begin_dir(p, calls[k], wait_other[k]);
+            int32_t rc = begin_dir(p, calls[k], wait_ev[k]);
             if (rc != KV_OK) return rc;
         }
         int32_t rc = issue_calls(p, calls, ncalls, false);

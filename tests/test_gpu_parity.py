@@ -316,3 +316,28 @@ def test_staged_transfer_planning_patterns(layout):
         assert st["device_status"] == 0 and st["kernel_launches"] > 0
     finally:
         p.close()
+
+
+@pytest.mark.parametrize("path", ["zerocopy", "staged"])
+def test_rotate_swap_in_waits_for_an_earlier_swap_out_that_reads_its_destinations(path):
+    """A long swap-out is still reading device blocks when a rotate arrives whose swap-in overwrites some
+    of them (the blocks were released in between).  The rotate's swap-in must follow the EARLIER
+    swap-out, not only the swap-out that travels in the same rotate."""
+    shape = W.KVShape(32, 16, 8, 128)             # 2 MiB blocks
+    nbg, nbh = 230, 420
+    p = _pair(shape, nbg, nbh, seed=13, path=PATHS[path])
+    try:
+        big_g = np.arange(0, 200, dtype=np.int32)
+        big_h = np.arange(0, 200, dtype=np.int32)
+        assert p.oracle.swap_out(big_g, big_h) == 0
+        og = np.arange(200, 210, dtype=np.int32)          # not part of the long swap-out
+        oh = np.arange(300, 310, dtype=np.int32)
+        ih = np.arange(400, 420, dtype=np.int32)          # untouched host blocks
+        ig = np.arange(180, 200, dtype=np.int32)          # the blocks the long swap-out reads last
+        r = W.Rotation(og, oh, ih, ig, np.zeros(1), np.zeros(1))
+        assert p.oracle.rotate(og, oh, ih, ig) == 0
+        assert p.pool.kv_swap_out(big_g, big_h) == 0      # 400 MiB over the link: several milliseconds
+        assert p.pool.kv_rotate(og, oh, ih, ig) == 0      # issued at once, no sync
+        p.assert_equal("rotate behind a long swap-out")
+    finally:
+        p.close()
