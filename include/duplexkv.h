@@ -53,7 +53,8 @@ extern "C" {
 #define KV_HOST_LAYER_FIRST   1
 
 /* transfer paths (how the host link is driven) */
-#define KV_PATH_AUTO          0     /* choice by bytes per block measured on B200 (see kv_path_for)      */
+#define KV_PATH_AUTO          0     /* per call: STAGED when the copy-engine transfers the call needs would
+                                       average 3 MiB or more, else ZEROCOPY (see kv_path_for)            */
 #define KV_PATH_ZEROCOPY      1     /* SM kernels read/write mapped pinned host memory directly          */
 #define KV_PATH_STAGED        2     /* pack kernel -> contiguous HBM staging -> copy engine (and reverse)*/
 #define KV_PATH_CE2D          3     /* one strided 2-D copy-engine transfer per block, no kernel         */
@@ -227,7 +228,9 @@ const char *kv_last_error(kv_pool_t *pool);
 int64_t kv_seg_bytes(int32_t block_size, int32_t kv_heads, int32_t head_dim);
 int64_t kv_blk_bytes(int32_t num_layers, int32_t block_size, int32_t kv_heads, int32_t head_dim);
 
-/* The path KV_PATH_AUTO resolves to for a block of blk_bytes (= kv_blk_bytes of the shape). */
+/* The path KV_PATH_AUTO resolves to for blocks of blk_bytes (= kv_blk_bytes of the shape) whose host ids
+ * have no neighbours in the list (such blocks travel two per transfer).  Lists with neighbouring host
+ * ids make larger transfers and can go STAGED at smaller block sizes; AUTO decides that per call. */
 int32_t kv_path_for(int64_t blk_bytes);
 
 /*

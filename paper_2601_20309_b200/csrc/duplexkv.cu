@@ -20,6 +20,7 @@ namespace {
 
 constexpr int KV_SLOTS = 8;            // descriptor / event ring depth per direction
 constexpr int KV_MAX_CE_STREAMS = 4;
+constexpr int64_t KV_AUTO_MIN_TRANSFER = 3ll << 20;   // AUTO: staged when its transfers average 3 MiB or more
 constexpr int BULK_STAGE = 16384;      // bytes per shared-memory stage of the bulk kernel
 constexpr int BULK_NS = 8;             // stages
 constexpr int BULK_AHEAD = 5;          // loads in flight ahead of the stores
@@ -288,18 +289,12 @@ struct DirCall {
     int path;
     // copy-engine issue state (CE paths are issued in slices so the two directions interleave)
     int64_t ce_next = 0;
+    bool planned = false;              // STAGED: plan_staged has run for this call
     int chunk_idx = 0;                 // STAGED: chunk being issued, next op of it
     int op_next = 0;
     bool chunk_open = false;
     unsigned rr = 0;                   // round-robin cursor over the direction's CE streams
 };
-
-int resolve_path(const kv_pool *p, int d)
-{
-    int path = p->dir[d].path;
-    if (path == KV_PATH_AUTO) path = kv_path_for(p->blk);
-    return path;
-}
 
 // fork: the extra streams of a CE direction wait for everything issued so far on its main stream
 int32_t ce_fork(kv_pool *p, DirState &s)
@@ -381,6 +376,7 @@ int32_t plan_staged(kv_pool *p, DirCall &c)
     } catch (...) {
         return fail(p, KV_ERR_NOMEM, "out of host memory");
     }
+    c.planned = true;
     return KV_OK;
 }
 
@@ -397,7 +393,6 @@ int32_t begin_dir(kv_pool *p, DirCall &c, cudaEvent_t wait_for)
     c.aux_dev = c.pairs_dev + p->cap;
     if (c.path == KV_PATH_STAGED) {
         if (!s.stage) {
-            s.half_blocks = std::max<int64_t>(1, p->cfg.staging_bytes / 2 / p->blk);
             cudaError_t e = cudaMalloc((void **)&s.stage, (size_t)(2 * s.half_blocks * p->blk));
             if (e != cudaSuccess) {
                 s.stage = nullptr;
@@ -405,8 +400,10 @@ int32_t begin_dir(kv_pool *p, DirCall &c, cudaEvent_t wait_for)
                 return fail(p, KV_ERR_NOMEM, "staging buffer allocation failed");
             }
         }
-        int32_t rc = plan_staged(p, c);
-        if (rc != KV_OK) return rc;
+        if (!c.planned) {
+            int32_t rc = plan_staged(p, c);
+            if (rc != KV_OK) return rc;
+        }
         // the kernel sees (device block id, position in the sorted list)
         for (int64_t k = 0; k < c.n; ++k) {
             const int32_t g = c.gpu_ids[s.order[(size_t)k]];
@@ -633,8 +630,25 @@ int32_t run_calls(kv_pool *p, DirCall *calls, int ncalls, const bool *wait_other
             const DirState &o = p->dir[1 - calls[k].d];
             wait_ev[k] = o.ev_end[o.issued % KV_SLOTS];
         }
+    // KV_PATH_AUTO is settled per call: plan the staged transfers first (cheap: a sort of the ids), and
+    // take the staged path when its transfers would carry KV_AUTO_MIN_TRANSFER bytes or more on average,
+    // the zero-copy kernels otherwise.  Both directions of a rotate take the same path (a kernel on one
+    // direction starves the copy engine on the other).
+    {
+        int64_t bytes = 0, ops = 0;
+        for (int k = 0; k < ncalls; ++k) {
+            calls[k].path = p->dir[calls[k].d].path;
+            if (calls[k].path != KV_PATH_AUTO) continue;
+            int32_t rc = plan_staged(p, calls[k]);
+            if (rc != KV_OK) return rc;
+            bytes += calls[k].n * p->blk;
+            ops += (int64_t)p->dir[calls[k].d].ops.size();
+        }
+        const int chosen = (ops > 0 && bytes >= ops * KV_AUTO_MIN_TRANSFER) ? KV_PATH_STAGED : KV_PATH_ZEROCOPY;
+        for (int k = 0; k < ncalls; ++k)
+            if (calls[k].path == KV_PATH_AUTO) calls[k].path = chosen;
+    }
     for (int k = 0; k < ncalls; ++k) {
-        calls[k].path = resolve_path(p, calls[k].d);
         if (fused && calls[k].d == 1) {
             // the fused launch runs on the out stream: order it after earlier swap-ins, and later swap-ins after it
             DirState &in = p->dir[1];
@@ -690,11 +704,13 @@ int64_t kv_blk_bytes(int32_t num_layers, int32_t block_size, int32_t kv_heads, i
 
 int32_t kv_path_for(int64_t blk_bytes)
 {
-    // Measured on B200 behind PCIe Gen5 x16, both directions busy, scattered ids: a copy-engine
-    // transfer costs a fixed start-up (about 10 us with the other direction busy) plus its bytes, so
-    // the staged path wins once its transfers (two blocks each when no host ids are neighbours) carry
-    // 4 MiB or more; below that the zero-copy kernels, which pay no per-block cost, are ahead.
-    return blk_bytes >= (2ll << 20) ? KV_PATH_STAGED : KV_PATH_ZEROCOPY;
+    // Measured on B200 behind PCIe Gen5 x16, both directions busy: a copy-engine transfer costs a fixed
+    // start-up (about 10 us with the other direction busy) plus its bytes, so the staged path wins once its
+    // transfers carry 3 MiB or more; below that the zero-copy kernels, which pay no per-transfer cost,
+    // are ahead.  Blocks with no neighbours in host memory travel two per transfer, hence this rule for
+    // fully scattered ids; a pool on KV_PATH_AUTO applies the same threshold to the transfers each call
+    // actually needs, so lists with neighbouring host ids go staged at any block size.
+    return 2 * blk_bytes >= KV_AUTO_MIN_TRANSFER ? KV_PATH_STAGED : KV_PATH_ZEROCOPY;
 }
 
 const char *kv_last_error(kv_pool_t *pool) { return pool ? pool->err : g_err; }
@@ -798,6 +814,7 @@ int32_t kv_pool_create(const kv_pool_config_t *cfg, kv_pool_t **out)
             KV_CREATE_CUDA(cudaEventCreate(&s.ev_end[k]));
         }
         s.ctas = want_ctas[d] > 0 ? want_ctas[d] : 64;
+        s.half_blocks = std::max<int64_t>(1, p->cfg.staging_bytes / 2 / blk);
         s.path = (d == 1 && cfg->path_in != KV_PATH_AUTO) ? cfg->path_in : cfg->path;
         s.nsub = cfg->ce_streams > 0 ? cfg->ce_streams : 1;
         s.sub[0] = s.stream;
@@ -941,8 +958,8 @@ int32_t kv_rotate(kv_pool_t *p, const int32_t *out_gpu, const int32_t *out_host,
         calls[1].n = n_in;
         const bool wait[2] = {conflicts_with_other(p, 0, out_gpu, out_host, n_out),
                               conflicts_with_other(p, 1, in_gpu, in_host, n_in)};
-        const bool fused = (p->cfg.flags & KV_FLAG_FUSED_ROTATE) && resolve_path(p, 0) == KV_PATH_ZEROCOPY &&
-                           resolve_path(p, 1) == KV_PATH_ZEROCOPY && !wait[0] && !wait[1];
+        const bool fused = (p->cfg.flags & KV_FLAG_FUSED_ROTATE) && p->dir[0].path == KV_PATH_ZEROCOPY &&
+                           p->dir[1].path == KV_PATH_ZEROCOPY && !wait[0] && !wait[1];
         return run_calls(p, calls, 2, wait, fused);
     }
     // overlap allowed: the conflict-free swap-ins run beside the swap-out, the others after it

@@ -67,7 +67,7 @@ def probe(out) -> None:
 
 
 PATHS = [("staged", B.KV_PATH_STAGED), ("zerocopy", B.KV_PATH_ZEROCOPY), ("ce2d", B.KV_PATH_CE2D),
-         ("naive", B.KV_PATH_NAIVE)]
+         ("naive", B.KV_PATH_NAIVE), ("auto", B.KV_PATH_AUTO)]
 
 
 def paths(out, max_payload_gb: float) -> None:
@@ -111,18 +111,19 @@ def paths(out, max_payload_gb: float) -> None:
                     t_b = best(lambda: pool.kv_rotate(rot.out_gpu, rot.out_host, rot.in_host, rot.in_gpu), reps)
                     rec[name] = {"out": round(nbytes / t_o / 1e6, 1), "in": round(nbytes / t_i / 1e6, 1),
                                  "both": round(2 * nbytes / t_b / 1e6, 1)}
+                    if name == "auto":
+                        rec["auto_took"] = B.PATH_NAMES[pool.kv_get_stats()["last_path_out"]]
                 pool.destroy()
                 del dev
                 torch.cuda.empty_cache()
-                rec["auto"] = B.PATH_NAMES[B.kv_path_for(shape.block_bytes)]
                 rows.append(rec)
                 _emit(rec, out)
     print("\n| block | BLK MiB | tables | payload MB | probe both | staged out/in/both | zero-copy out/in/both | "
-          "2-D per block out/in/both | per segment out/in/both | AUTO |\n|---|---|---|---|---|---|---|---|---|---|")
+          "2-D per block out/in/both | per segment out/in/both | AUTO out/in/both | AUTO took |\n|---|---|---|---|---|---|---|---|---|---|---|")
     for r in rows:
         f = lambda k: "%s / %s / %s" % (r[k]["out"], r[k]["in"], r[k]["both"]) if k in r else "-"
         print(f"| {r['block_size']} | {r['blk_mib']:g} | {r['tables']} | {r['payload_mb']} | {r['probe_bi_gbs']} | "
-              f"{f('staged')} | {f('zerocopy')} | {f('ce2d')} | {f('naive')} | {r['auto']} |")
+              f"{f('staged')} | {f('zerocopy')} | {f('ce2d')} | {f('naive')} | {f('auto')} | {r['auto_took']} |")
 
 
 def main() -> None:
