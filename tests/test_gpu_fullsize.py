@@ -69,13 +69,16 @@ def test_config2_full_size_rotate_single_swaps_and_pairwise_rotations():
         for _ in range(2):                                      # the bench repeats this very call
             assert tags.rotate(rot.out_gpu.tolist(), rot.out_host.tolist(), rot.in_host.tolist(), rot.in_gpu.tolist()) == 0
             assert pool.kv_rotate(rot.out_gpu, rot.out_host, rot.in_host, rot.in_gpu) == 0
-        for r in w.extra["pairs"]:
+        pool.kv_sync()
+        st = pool.kv_get_stats()
+        assert B.PATH_NAMES[st["last_path_out"]] == "staged" and B.PATH_NAMES[st["last_path_in"]] == "staged"
+        assert st["timed_kernels"] > 0                          # the bench's path and kernels ran
+        for r in w.extra["pairs"]:                              # small ones may take the zero-copy kernels
             assert tags.rotate(r.out_gpu.tolist(), r.out_host.tolist(), r.in_host.tolist(), r.in_gpu.tolist()) == 0
             assert pool.kv_rotate(r.out_gpu, r.out_host, r.in_host, r.in_gpu) == 0
         pool.kv_sync()
         st = pool.kv_get_stats()
         assert st["device_status"] == 0
-        assert B.PATH_NAMES[st["last_path_out"]] == "staged" and st["timed_kernels"] > 0     # the bench's path ran
 
         d1 = {W.POOL_GPU: F.checksum_blocks(lay_g, nb_gpu), W.POOL_HOST: F.checksum_blocks(lay_h, nb_host)}
         g_origin = np.array(tags.g_tag, dtype=np.int64)         # (origin pool, origin block) per slot
