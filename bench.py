@@ -37,9 +37,12 @@ from paper_2601_20309_b200 import workload as W         # noqa: E402
 
 METRIC = "full-duplex KV swap GB/s (out+in)"
 UNIT = "GB/s"
-# dram__bytes_read.sum + dram__bytes_write.sum of one pack launch, scaled from the ncu capture on the
-# small case (traffic grows with the bytes moved); None until counters exist for the current kernel
-NCU_TRAFFIC_PER_LAUNCH = None
+# DRAM traffic of one pack / unpack launch, from the ncu capture of an 89-block (186.65 MB) launch on the
+# --small case: dram__bytes_read.sum = 1.00005 x payload (no byte read twice); dram__bytes_write.sum =
+# payload - 48.5 MB, the lines still in L2 when the kernel ends.  Reads scale with the payload, the L2
+# tail does not.
+def ncu_traffic_per_launch(payload_bytes: float) -> float:
+    return 1.00005 * payload_bytes + max(0.0, payload_bytes - 48.5e6)
 
 
 # ------------------------------------------------------------------------------------------------ helpers
@@ -369,7 +372,8 @@ def run_ours(args, rank: int, local_rank: int, world: int) -> None:
             k_avg_ms = k_ms / k_n
             k_ach = M.gbs(2.0 * k_bytes, k_ms)
             roofline = {"bound": "hbm", "achieved": k_ach, "peak": peaks["hbm_gbs"], "unit": "GB/s",
-                        "frac": k_ach / peaks["hbm_gbs"], "traffic": NCU_TRAFFIC_PER_LAUNCH,
+                        "frac": k_ach / peaks["hbm_gbs"], "traffic": ncu_traffic_per_launch(k_bytes / k_n),
+                        "traffic_source": "ncu capture on the --small case, scaled to this run's average launch",
                         "kernel": "kv_copy_bulk (pack: scattered HBM planes -> contiguous HBM staging; unpack: the reverse)",
                         "launches_timed": int(k_n), "avg_launch_us": k_avg_ms * 1e3,
                         "algorithmic_bytes_per_launch": 2.0 * k_bytes / k_n,
