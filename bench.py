@@ -194,11 +194,7 @@ def run_ours(args, rank: int, local_rank: int, world: int) -> None:
         torch.cuda.synchronize()
 
     def reduce(x: float, op: str) -> float:
-        if dist is None:
-            return x
-        t = torch.tensor([x], dtype=torch.float64, device=dev)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX if op == "max" else dist.ReduceOp.SUM)
-        return float(t.item())
+        return M.reduce_over_ranks(x, op, dist, dev)
 
     # ---- host-link denominators, measured in this process (again after the timed region)
     probe = B.kv_probe_link(local_rank, 256 << 20, 4)

@@ -42,3 +42,22 @@ def percentile(xs: Sequence[float], q: float) -> float:
 
 def median(xs: Iterable[float]) -> float:
     return statistics.median(list(xs))
+
+
+def reduce_over_ranks(x: float, op: str, dist=None, device: str = "cpu") -> float:
+    """Maximum or sum of a per-rank number over the ranks of an initialised ``torch.distributed`` group
+    (``dist`` is the module; ``None`` = single process).  Replicas are timed as the slowest rank and
+    their bytes are added: job GB/s = sum of bytes / max of time."""
+    if dist is None:
+        return float(x)
+    import torch
+    t = torch.tensor([x], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX if op == "max" else dist.ReduceOp.SUM)
+    return float(t.item())
+
+
+def replicas_gbs(bytes_per_rank: float, ms_per_rank: float, dist=None, device: str = "cpu") -> float:
+    """Whole-job GB/s of independent replicas: every rank's bytes over the slowest rank's time."""
+    total = reduce_over_ranks(bytes_per_rank, "sum", dist, device)
+    slowest = reduce_over_ranks(ms_per_rank, "max", dist, device)
+    return gbs(total, slowest)

@@ -1,0 +1,52 @@
+"""The multi-GPU mode is independent replicas: no exchange on the data path, only the aggregation of the
+per-rank figures (bytes are added, time is the slowest rank's).  Checked here with two gloo ranks on CPU."""
+import os
+import socket
+
+import pytest
+import torch
+import torch.distributed as dist
+import torch.multiprocessing as mp
+
+from paper_2601_20309_b200 import metrics as M
+
+
+def _free_port():
+    with socket.socket() as s:
+        s.bind(("127.0.0.1", 0))
+        return s.getsockname()[1]
+
+
+def _rank(rank, world, port, q):
+    os.environ["MASTER_ADDR"] = "127.0.0.1"
+    os.environ["MASTER_PORT"] = str(port)
+    dist.init_process_group("gloo", rank=rank, world_size=world)
+    try:
+        nbytes = 7.0e9 + rank * 1.0e9            # rank 0 moved 7 GB, rank 1 moved 8 GB
+        ms = 100.0 + 50.0 * rank                 # rank 1 is the slow one
+        q.put((rank, M.reduce_over_ranks(nbytes, "sum", dist), M.reduce_over_ranks(ms, "max", dist),
+               M.replicas_gbs(nbytes, ms, dist)))
+        dist.barrier()
+    finally:
+        dist.destroy_process_group()
+
+
+def test_two_replicas_add_bytes_and_take_the_slowest_time():
+    world, port = 2, _free_port()
+    ctx = mp.get_context("spawn")
+    q = ctx.Queue()
+    procs = [ctx.Process(target=_rank, args=(r, world, port, q)) for r in range(world)]
+    for p in procs:
+        p.start()
+    got = [q.get(timeout=120) for _ in range(world)]
+    for p in procs:
+        p.join(timeout=60)
+        assert p.exitcode == 0
+    for _, total, slowest, gbs in got:
+        assert total == 15.0e9 and slowest == 150.0
+        assert gbs == pytest.approx(15.0e9 / 0.150 / 1e9)
+
+
+def test_single_process_is_the_identity():
+    assert M.reduce_over_ranks(3.5, "max") == 3.5
+    assert M.replicas_gbs(2e9, 1000.0) == pytest.approx(2.0)
