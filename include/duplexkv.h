@@ -259,6 +259,95 @@ typedef struct {
 } kv_probe_spec_t;
 int32_t kv_probe_link_ex(int32_t device_id, const kv_probe_spec_t *spec, kv_link_probe_t *out);
 
+/* Shape of a pool (what kv_pool_create was given). */
+typedef struct {
+    int32_t num_layers, block_size, kv_heads, head_dim;
+    int64_t num_gpu_blocks, num_host_blocks, seg_bytes, blk_bytes;
+} kv_pool_shape_t;
+int32_t kv_pool_shape(kv_pool_t *pool, kv_pool_shape_t *out);
+
+/* Calls issued and calls known to have completed, per direction (a non-blocking look at the pool's
+ * end events).  Any pointer may be NULL.  kv_gather_blocks / kv_scatter_blocks count as calls of the
+ * out / in direction. */
+int32_t kv_pool_progress(kv_pool_t *pool, int64_t *out_issued, int64_t *out_done, int64_t *in_issued, int64_t *in_done);
+
+/* ------------------------------------------------------------------------------------------------
+ * Block table with eager block rotation (section 4.3.2, "Eager block rotation for data race free
+ * overlapping", and the block table of the architecture figure in section 4.1).
+ *
+ * The table owns the free lists of both pools and, per request, the device block, host block and
+ * state of every block.  A block that is completely filled never changes again; once it has a copy
+ * in host memory it is "synced".  kv_eager_rotate copies full blocks to host memory in the
+ * background; kv_req_rotate preempts and resumes whole requests with ONE kv_rotate on the pool,
+ * moving out only the blocks that have no valid host copy (normally the single, partly filled
+ * "dirty" block) and releasing the others' device blocks without any transfer, so that the requests
+ * resuming in the same call can take them: the swap-in never depends on the swap-out.  Host copies
+ * are kept while a request runs on the GPU.  Host blocks are handed out in runs, so blocks sent
+ * together are neighbours in host memory and travel as few, long transfers.
+ *
+ * All calls return a status like the pool's; data movement is asynchronous (kv_sync on the pool
+ * waits for it).  One caller thread.  The table does not write KV data: whoever runs the model
+ * writes tokens into the device blocks kv_req_blocks reports.  Device blocks handed out by kv_req_add
+ * and kv_req_append are never still being read by a swap-out (blocks released at a preemption are
+ * held back until the copies that may read them have finished; the call waits for the pool if it
+ * must), so the caller may write into them at once.  A host block released by kv_req_finish, and the
+ * host pool in general, is only ever written by the pool's own swap-outs, which the pool orders.
+ * Request ids are arbitrary int64 values chosen by the caller.
+ */
+typedef struct kv_table kv_table_t;
+
+typedef struct {
+    int64_t tokens, num_blocks;
+    int64_t synced_blocks;      /* blocks whose host copy is valid                                   */
+    int64_t host_blocks;        /* blocks that own a host block (valid or stale)                     */
+    int64_t dirty_blocks;       /* partly filled blocks: 0 or 1 (the last one)                        */
+    int32_t on_gpu, pad_;       /* 1 = runs on the GPU, 0 = preempted (lives in host memory)          */
+} kv_req_info_t;
+
+typedef struct {
+    int64_t eager_blocks, eager_calls;          /* blocks copied out in the background, calls that did */
+    int64_t preempt_blocks_moved;               /* blocks copied out at preemption time                */
+    int64_t discarded_blocks;                   /* device blocks released at preemption without a copy */
+    int64_t resume_blocks_moved;                /* blocks copied in at resume time                     */
+    int64_t preempted_requests, resumed_requests, rotate_calls;
+    int64_t free_gpu_blocks, free_host_blocks, free_host_extents, requests;
+} kv_table_stats_t;
+
+/* A table over `pool` (borrowed; destroy the table first).  Every block of both pools starts free. */
+int32_t kv_table_create(kv_pool_t *pool, kv_table_t **out);
+/* The same bookkeeping with no pool behind it: nothing is moved.  For planning and for testing the
+ * allocator and the state machine on a machine without a GPU. */
+int32_t kv_table_create_dry(int64_t num_gpu_blocks, int64_t num_host_blocks, int32_t block_size, kv_table_t **out);
+int32_t kv_table_destroy(kv_table_t *table);
+const char *kv_table_last_error(kv_table_t *table);
+
+/* New request on the GPU whose first `tokens` tokens are about to be written (prefill): takes
+ * ceil(tokens/block_size) device blocks.  KV_ERR_NOMEM (nothing changed) when they are not free. */
+int32_t kv_req_add(kv_table_t *table, int64_t req, int64_t tokens);
+/* `new_tokens` more tokens for a request on the GPU (decode): they go into the partly filled last
+ * block first (its host copy, if any, becomes stale), then into newly taken device blocks. */
+int32_t kv_req_append(kv_table_t *table, int64_t req, int64_t new_tokens);
+/* Background step: copy up to max_blocks full blocks that have no valid host copy to host memory
+ * (requests in arrival order, round robin across calls) with one kv_swap_out, and mark them synced.
+ * *n_issued (may be NULL) = blocks sent.  Sends fewer when the host pool runs out. */
+int32_t kv_eager_rotate(kv_table_t *table, int64_t max_blocks, int64_t *n_issued);
+/* Preempt the listed requests (HOST array of ids; must be on the GPU) and resume the listed ones
+ * (must be preempted) in one full-duplex kv_rotate.  All or nothing: KV_ERR_NOMEM / KV_ERR_INVALID_ARG
+ * leave the table unchanged. */
+int32_t kv_req_rotate(kv_table_t *table, const int64_t *preempt, int64_t n_preempt,
+                      const int64_t *resume, int64_t n_resume);
+int32_t kv_req_preempt(kv_table_t *table, int64_t req);
+int32_t kv_req_resume(kv_table_t *table, int64_t req);
+/* The request is done: all its device and host blocks become free. */
+int32_t kv_req_finish(kv_table_t *table, int64_t req);
+
+int32_t kv_req_info(kv_table_t *table, int64_t req, kv_req_info_t *out);
+/* Per block, in logical order: device id (-1 = none), host id (-1 = none), whether the host copy is
+ * valid.  Output arrays are HOST memory of at least `cap` >= num_blocks entries; any may be NULL. */
+int32_t kv_req_blocks(kv_table_t *table, int64_t req, int32_t *gpu_ids, int32_t *host_ids,
+                      uint8_t *host_valid, int64_t cap);
+int32_t kv_table_get_stats(kv_table_t *table, kv_table_stats_t *out);
+
 #ifdef __cplusplus
 }
 #endif

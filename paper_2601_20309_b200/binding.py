@@ -70,10 +70,31 @@ class kv_probe_spec_t(C.Structure):
                 ("rows", C.c_int64), ("host_pitch", C.c_int64), ("dev_pitch", C.c_int64)]
 
 
+class kv_pool_shape_t(C.Structure):
+    _fields_ = [("num_layers", C.c_int32), ("block_size", C.c_int32), ("kv_heads", C.c_int32), ("head_dim", C.c_int32),
+                ("num_gpu_blocks", C.c_int64), ("num_host_blocks", C.c_int64), ("seg_bytes", C.c_int64),
+                ("blk_bytes", C.c_int64)]
+
+
+class kv_req_info_t(C.Structure):
+    _fields_ = [("tokens", C.c_int64), ("num_blocks", C.c_int64), ("synced_blocks", C.c_int64),
+                ("host_blocks", C.c_int64), ("dirty_blocks", C.c_int64), ("on_gpu", C.c_int32), ("pad_", C.c_int32)]
+
+
+class kv_table_stats_t(C.Structure):
+    _fields_ = [(n, C.c_int64) for n in ("eager_blocks", "eager_calls", "preempt_blocks_moved", "discarded_blocks",
+                                         "resume_blocks_moved", "preempted_requests", "resumed_requests",
+                                         "rotate_calls", "free_gpu_blocks", "free_host_blocks", "free_host_extents",
+                                         "requests")]
+
+
 EXPORTS = ["kv_pool_create", "kv_pool_destroy", "kv_pool_set_path", "kv_swap_out", "kv_swap_in", "kv_rotate", "kv_sync",
            "kv_gather_blocks", "kv_scatter_blocks", "kv_host_ptr", "kv_get_stats", "kv_last_error",
            "kv_seg_bytes", "kv_blk_bytes", "kv_path_for", "kv_probe_link", "kv_probe_link_ex",
-           "kv_gather_blocks_static"]
+           "kv_gather_blocks_static", "kv_pool_shape", "kv_pool_progress",
+           "kv_table_create", "kv_table_create_dry", "kv_table_destroy", "kv_table_last_error", "kv_req_add",
+           "kv_req_append", "kv_eager_rotate", "kv_req_rotate", "kv_req_preempt", "kv_req_resume", "kv_req_finish",
+           "kv_req_info", "kv_req_blocks", "kv_table_get_stats"]
 
 _lib = None
 
@@ -118,6 +139,36 @@ def lib() -> C.CDLL:
     L.kv_path_for.argtypes = [i64]
     L.kv_probe_link.restype = C.c_int32
     L.kv_probe_link.argtypes = [C.c_int32, i64, C.c_int32, C.POINTER(kv_link_probe_t)]
+    i64p = C.POINTER(C.c_int64)
+    L.kv_pool_shape.restype = C.c_int32
+    L.kv_pool_shape.argtypes = [vp, C.POINTER(kv_pool_shape_t)]
+    L.kv_pool_progress.restype = C.c_int32
+    L.kv_pool_progress.argtypes = [vp, i64p, i64p, i64p, i64p]
+    L.kv_table_create.restype = C.c_int32
+    L.kv_table_create.argtypes = [vp, C.POINTER(vp)]
+    L.kv_table_create_dry.restype = C.c_int32
+    L.kv_table_create_dry.argtypes = [i64, i64, C.c_int32, C.POINTER(vp)]
+    L.kv_table_destroy.restype = C.c_int32
+    L.kv_table_destroy.argtypes = [vp]
+    L.kv_table_last_error.restype = C.c_char_p
+    L.kv_table_last_error.argtypes = [vp]
+    L.kv_req_add.restype = C.c_int32
+    L.kv_req_add.argtypes = [vp, i64, i64]
+    L.kv_req_append.restype = C.c_int32
+    L.kv_req_append.argtypes = [vp, i64, i64]
+    L.kv_eager_rotate.restype = C.c_int32
+    L.kv_eager_rotate.argtypes = [vp, i64, i64p]
+    L.kv_req_rotate.restype = C.c_int32
+    L.kv_req_rotate.argtypes = [vp, i64p, i64, i64p, i64]
+    for name in ("kv_req_preempt", "kv_req_resume", "kv_req_finish"):
+        getattr(L, name).restype = C.c_int32
+        getattr(L, name).argtypes = [vp, i64]
+    L.kv_req_info.restype = C.c_int32
+    L.kv_req_info.argtypes = [vp, i64, C.POINTER(kv_req_info_t)]
+    L.kv_req_blocks.restype = C.c_int32
+    L.kv_req_blocks.argtypes = [vp, i64, i32p, i32p, C.POINTER(C.c_uint8), i64]
+    L.kv_table_get_stats.restype = C.c_int32
+    L.kv_table_get_stats.argtypes = [vp, C.POINTER(kv_table_stats_t)]
     L.kv_gather_blocks_static.restype = C.c_int32
     L.kv_gather_blocks_static.argtypes = [vp, C.c_int32, C.c_int32, C.c_int32, C.c_int32, i64, i32p, i64, vp, vp]
     L.kv_probe_link_ex.restype = C.c_int32
@@ -287,8 +338,95 @@ class KVPool:
     def kv_last_error(self) -> str:
         return lib().kv_last_error(self._h).decode()
 
+    def kv_pool_progress(self) -> dict:
+        v = [C.c_int64() for _ in range(4)]
+        self._ret(lib().kv_pool_progress(self._h, *[C.byref(x) for x in v]), True)
+        return dict(zip(("out_issued", "out_done", "in_issued", "in_done"), (x.value for x in v)))
+
+    def kv_pool_shape(self) -> dict:
+        sh = kv_pool_shape_t()
+        self._ret(lib().kv_pool_shape(self._h, C.byref(sh)), True)
+        return {k: getattr(sh, k) for k, _ in kv_pool_shape_t._fields_}
+
     # -- convenience for verification (no data path): the host pool as a numpy view
     def host_array(self) -> np.ndarray:
         base, nbytes = self.kv_host_ptr()
         buf = (C.c_uint8 * nbytes).from_address(base)
         return np.frombuffer(buf, dtype=np.uint8)
+
+
+class KVTable:
+    """Thin owner of a ``kv_table_t*`` (block table with eager block rotation).  ``pool`` is a ``KVPool`` or,
+    for bookkeeping without a GPU, ``None`` with the sizes given.  Methods return the C status unless
+    ``check`` (default) turns a negative one into ``KVError``."""
+
+    def __init__(self, pool: Optional[KVPool] = None, *, num_gpu_blocks: int = 0, num_host_blocks: int = 0,
+                 block_size: int = 0):
+        self._h = C.c_void_p()
+        self.pool = pool
+        if pool is not None:
+            rc = lib().kv_table_create(pool._h, C.byref(self._h))
+        else:
+            rc = lib().kv_table_create_dry(num_gpu_blocks, num_host_blocks, block_size, C.byref(self._h))
+        if rc != KV_OK:
+            raise KVError(rc, "kv_table_create failed")
+
+    def destroy(self) -> None:
+        if self._h:
+            lib().kv_table_destroy(self._h)
+            self._h = C.c_void_p()
+
+    def __del__(self):
+        try:
+            self.destroy()
+        except Exception:
+            pass
+
+    def _ret(self, rc: int, check: bool) -> int:
+        if check and rc != KV_OK:
+            raise KVError(rc, lib().kv_table_last_error(self._h).decode())
+        return rc
+
+    def kv_req_add(self, req: int, tokens: int, check: bool = True) -> int:
+        return self._ret(lib().kv_req_add(self._h, req, tokens), check)
+
+    def kv_req_append(self, req: int, new_tokens: int, check: bool = True) -> int:
+        return self._ret(lib().kv_req_append(self._h, req, new_tokens), check)
+
+    def kv_eager_rotate(self, max_blocks: int) -> int:
+        n = C.c_int64()
+        self._ret(lib().kv_eager_rotate(self._h, max_blocks, C.byref(n)), True)
+        return n.value
+
+    def kv_req_rotate(self, preempt: Sequence[int], resume: Sequence[int], check: bool = True) -> int:
+        p = (C.c_int64 * len(preempt))(*preempt)
+        r = (C.c_int64 * len(resume))(*resume)
+        return self._ret(lib().kv_req_rotate(self._h, p, len(preempt), r, len(resume)), check)
+
+    def kv_req_preempt(self, req: int, check: bool = True) -> int:
+        return self._ret(lib().kv_req_preempt(self._h, req), check)
+
+    def kv_req_resume(self, req: int, check: bool = True) -> int:
+        return self._ret(lib().kv_req_resume(self._h, req), check)
+
+    def kv_req_finish(self, req: int, check: bool = True) -> int:
+        return self._ret(lib().kv_req_finish(self._h, req), check)
+
+    def kv_req_info(self, req: int) -> dict:
+        out = kv_req_info_t()
+        self._ret(lib().kv_req_info(self._h, req, C.byref(out)), True)
+        return {k: getattr(out, k) for k, _ in kv_req_info_t._fields_ if k != "pad_"}
+
+    def kv_req_blocks(self, req: int):
+        """(device ids, host ids, host_valid) as numpy arrays; -1 where a block has no id."""
+        n = self.kv_req_info(req)["num_blocks"]
+        g, h, v = np.empty(n, np.int32), np.empty(n, np.int32), np.empty(n, np.uint8)
+        i32p = C.POINTER(C.c_int32)
+        self._ret(lib().kv_req_blocks(self._h, req, g.ctypes.data_as(i32p), h.ctypes.data_as(i32p),
+                                      v.ctypes.data_as(C.POINTER(C.c_uint8)), n), True)
+        return g, h, v.astype(bool)
+
+    def kv_table_get_stats(self) -> dict:
+        out = kv_table_stats_t()
+        self._ret(lib().kv_table_get_stats(self._h, C.byref(out)), True)
+        return {k: getattr(out, k) for k, _ in kv_table_stats_t._fields_}

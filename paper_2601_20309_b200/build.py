@@ -1,7 +1,7 @@
 """Compile the CUDA library for sm_100a with nvcc, in-tree.
 
 ``build()`` produces ``paper_2601_20309_b200/libduplexkv.so`` from ``csrc/duplexkv.cu``
-(kernels in ``csrc/kv_kernels.cuh``) and ``libkvtestutil.so`` from ``csrc/kv_testutil.cu``
+(kernels in ``csrc/kv_kernels.cuh``) and ``csrc/kv_table.cu`` (block table, host code) and ``libkvtestutil.so`` from ``csrc/kv_testutil.cu``
 (pool fill / checksum helpers used by tests and the bench to make and check inputs; not
 part of the rotation path).  nvcc cross-compiles without a GPU.
 """
@@ -35,16 +35,17 @@ def _stale(target: str, sources) -> bool:
 
 
 def build(force: bool = False, verbose: bool = False) -> str:
-    main_src = [os.path.join(CSRC, "duplexkv.cu"), os.path.join(CSRC, "kv_kernels.cuh"),
-                os.path.join(os.path.dirname(HERE), "include", "duplexkv.h")]
-    jobs = [(LIB, main_src)]
+    # (target, files to compile, further files the target depends on)
+    main_src = [os.path.join(CSRC, "duplexkv.cu"), os.path.join(CSRC, "kv_table.cu")]
+    main_dep = [os.path.join(CSRC, "kv_kernels.cuh"), os.path.join(os.path.dirname(HERE), "include", "duplexkv.h")]
+    jobs = [(LIB, main_src, main_dep)]
     util_src = os.path.join(CSRC, "kv_testutil.cu")
     if os.path.exists(util_src):
-        jobs.append((TESTUTIL_LIB, [util_src]))
-    for target, sources in jobs:
-        if not force and not _stale(target, sources):
+        jobs.append((TESTUTIL_LIB, [util_src], []))
+    for target, sources, deps in jobs:
+        if not force and not _stale(target, sources + deps):
             continue
-        cmd = [_nvcc()] + NVCC_FLAGS + (["-Xptxas", "-v"] if verbose else []) + ["-o", target, sources[0]]
+        cmd = [_nvcc()] + NVCC_FLAGS + (["-Xptxas", "-v"] if verbose else []) + ["-o", target] + sources
         res = subprocess.run(cmd, capture_output=True, text=True)
         if verbose:
             sys.stderr.write(res.stderr)

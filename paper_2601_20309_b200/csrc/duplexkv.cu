@@ -1119,6 +1119,31 @@ int32_t kv_scatter_blocks(kv_pool_t *p, const void *src_device, const int32_t *g
     return device_leg(p, gpu_ids, n, src_device, 1);
 }
 
+int32_t kv_pool_progress(kv_pool_t *p, int64_t *out_issued, int64_t *out_done, int64_t *in_issued, int64_t *in_done)
+{
+    if (!p) return KV_ERR_INVALID_ARG;
+    poll_done(p);
+    if (out_issued) *out_issued = (int64_t)p->dir[0].issued;
+    if (out_done) *out_done = (int64_t)p->dir[0].done;
+    if (in_issued) *in_issued = (int64_t)p->dir[1].issued;
+    if (in_done) *in_done = (int64_t)p->dir[1].done;
+    return KV_OK;
+}
+
+int32_t kv_pool_shape(kv_pool_t *p, kv_pool_shape_t *out)
+{
+    if (!p || !out) return KV_ERR_INVALID_ARG;
+    out->num_layers = p->cfg.num_layers;
+    out->block_size = p->cfg.block_size;
+    out->kv_heads = p->cfg.kv_heads;
+    out->head_dim = p->cfg.head_dim;
+    out->num_gpu_blocks = p->cfg.num_gpu_blocks;
+    out->num_host_blocks = p->cfg.num_host_blocks;
+    out->seg_bytes = p->seg;
+    out->blk_bytes = p->blk;
+    return KV_OK;
+}
+
 int32_t kv_host_ptr(kv_pool_t *p, void **base, int64_t *bytes)
 {
     if (!p || !base || !bytes) return KV_ERR_INVALID_ARG;
