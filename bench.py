@@ -303,6 +303,33 @@ def run_ours(args, rank: int, local_rank: int, world: int) -> None:
         t_c = timed(lambda: pool.kv_rotate(og, oh_c, ih_c, ig))
         contiguous_host = M.gbs(bytes_out + bytes_in, t_c)
         F.fill_blocks(F.Layout.host(host_base, shape, nb_host), w.seed, W.POOL_HOST, len(og), device=dev)   # restore what it overwrote
+        # ---- the same 16 + 16 requests through the block table (run-based host ids, eager block rotation)
+        table = B.KVTable(pool)
+        len_a = np.diff(rot.out_req_offsets).astype(int)
+        len_b = np.diff(rot.in_req_offsets).astype(int)
+        ids_a, ids_b = list(range(len(len_a))), list(range(100, 100 + len(len_b)))
+        for rid, nb in zip(ids_a + ids_b, list(len_a) + list(len_b)):
+            table.kv_req_add(rid, int(nb) * shape.block_size - 5)          # last block partly filled
+        table.kv_req_rotate(ids_b, [])                                      # B leaves the GPU: everything is sent
+        pool.kv_sync()
+
+        def table_rotate(pre, res):
+            s0, p0 = table.kv_table_get_stats(), pool.kv_get_stats()
+            table.kv_req_rotate(pre, res)
+            pool.kv_sync()
+            s1, p1 = table.kv_table_get_stats(), pool.kv_get_stats()
+            nbytes = (p1["bytes_out"] - p0["bytes_out"]) + (p1["bytes_in"] - p0["bytes_in"])
+            return {"ms": p1["last_union_ms"], "gbs": M.gbs(nbytes, p1["last_union_ms"]),
+                    "blocks_out": s1["preempt_blocks_moved"] - s0["preempt_blocks_moved"],
+                    "blocks_discarded": s1["discarded_blocks"] - s0["discarded_blocks"],
+                    "blocks_in": s1["resume_blocks_moved"] - s0["resume_blocks_moved"]}
+        tb = {}
+        tb["rotate_nothing_copied_beforehand"] = table_rotate(ids_a, ids_b)    # A out (all blocks), B in
+        tb["rotate_back_host_copies_still_valid"] = table_rotate(ids_b, ids_a)  # B out (nothing to send), A in
+        for rid in ids_a:
+            table.kv_req_append(rid, 1)                                        # A generated a token each
+        tb["rotate_after_one_token_each"] = table_rotate(ids_a, ids_b)          # A out (one dirty block each), B in
+        table.destroy()
         # ---- single swaps of the median-length and the longest request
         singles = {}
         for key, which in (("single_out", "out"), ("single_in", "in")):
@@ -335,7 +362,7 @@ def run_ours(args, rank: int, local_rank: int, world: int) -> None:
         leg_bytes = 2.0 * len(og) * shape.block_bytes          # read + write
         del stage
         extra = {"paths": paths, "singles": singles, "lat_us": lat_us, "lat_blocks": lat_blocks, "leg": leg,
-                 "leg_bytes": leg_bytes, "probe2": probe2, "contiguous_host": contiguous_host}
+                 "leg_bytes": leg_bytes, "probe2": probe2, "contiguous_host": contiguous_host, "table": tb}
 
     pool.destroy()
     del device_pool
@@ -413,6 +440,7 @@ def run_ours(args, rank: int, local_rank: int, world: int) -> None:
                            "e2e_ms_serial_u": uni["e2e_ms_serial_u"], "e2e_ms_concurrent_b": step_ms},
             "paths_on_same_lists": paths,
             "rotate_with_neighbouring_host_ids_gbs": extra["contiguous_host"],
+            "block_table": extra["table"],
             "single_swaps": extra["singles"],
             "request_rotate_us": {"p50": M.percentile(extra["lat_us"], 0.5), "p99": M.percentile(extra["lat_us"], 0.99),
                                   "n": len(extra["lat_us"]),
