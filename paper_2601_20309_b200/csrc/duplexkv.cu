@@ -24,6 +24,11 @@ constexpr int64_t KV_AUTO_MIN_TRANSFER = 3ll << 20;   // AUTO: staged when its t
 constexpr int BULK_STAGE = 16384;      // bytes per shared-memory stage of the bulk kernel
 constexpr int BULK_NS = 8;             // stages
 constexpr int BULK_AHEAD = 5;          // loads in flight ahead of the stores
+// the same kernel when one side is mapped host memory: the link needs far fewer bytes in flight than
+// HBM does, and a small shared-memory footprint leaves the SMs' L1 to whatever else runs on them
+constexpr int LINK_STAGE = 8192;
+constexpr int LINK_NS = 8;
+constexpr int LINK_AHEAD = 6;
 constexpr int LDST_THREADS = 512;
 constexpr int LDST_UNROLL = 4;         // 512 threads * 4 * 16 B = 32 KiB per item
 constexpr int LDST_CHUNK = LDST_THREADS * LDST_UNROLL * 16;
@@ -145,9 +150,9 @@ KvSide packed_side(const kv_pool *p, const void *base)
 
 bool use_ldst(const kv_pool *p) { return (p->cfg.flags & KV_FLAG_LDST_KERNEL) != 0; }
 
-void fill_geometry(const kv_pool *p, KvJob &job)
+void fill_geometry(const kv_pool *p, KvJob &job, bool link = false)
 {
-    const int max_chunk = use_ldst(p) ? LDST_CHUNK : BULK_STAGE;
+    const int max_chunk = use_ldst(p) ? LDST_CHUNK : (link ? LINK_STAGE : BULK_STAGE);
     job.planes = p->planes;
     job.seg = (int)p->seg;
     job.chunk = (int)std::min<int64_t>(p->seg, max_chunk);
@@ -161,12 +166,14 @@ int clamp_ctas(const KvJob &job, const KvDir &d, int want)
     return (int)std::max<long long>(1, std::min<long long>(want, items));
 }
 
-cudaError_t launch_job(kv_pool *p, const KvJob &job, cudaStream_t stream)
+cudaError_t launch_job(kv_pool *p, const KvJob &job, cudaStream_t stream, bool link = false)
 {
     const int grid = job.dir[0].ctas + job.dir[1].ctas;
     if (grid <= 0) return cudaSuccess;
     if (use_ldst(p)) {
         kv_copy_ldst<LDST_THREADS, LDST_UNROLL><<<grid, LDST_THREADS, 0, stream>>>(job);
+    } else if (link) {
+        kv_copy_bulk<LINK_STAGE, LINK_NS, LINK_AHEAD><<<grid, 32, LINK_STAGE * LINK_NS, stream>>>(job);
     } else {
         kv_copy_bulk<BULK_STAGE, BULK_NS, BULK_AHEAD><<<grid, 32, BULK_STAGE * BULK_NS, stream>>>(job);
     }
@@ -586,23 +593,23 @@ int32_t issue_calls(kv_pool *p, DirCall *calls, int ncalls, bool fused)
     // kernel (zero-copy) directions
     if (fused && ncalls == 2 && calls[0].path == KV_PATH_ZEROCOPY && calls[1].path == KV_PATH_ZEROCOPY) {
         KvJob job;
-        fill_geometry(p, job);
+        fill_geometry(p, job, true);
         job.dir[0] = zerocopy_dir(p, calls[0]);
         job.dir[1] = zerocopy_dir(p, calls[1]);
         job.dir[0].ctas = clamp_ctas(job, job.dir[0], p->dir[0].ctas);
         job.dir[1].ctas = clamp_ctas(job, job.dir[1], p->dir[1].ctas);
-        KV_CUDA(p, launch_job(p, job, p->dir[0].stream));
+        KV_CUDA(p, launch_job(p, job, p->dir[0].stream, true));
         return KV_OK;
     }
     for (int k = 0; k < ncalls; ++k) {
         DirCall &c = calls[k];
         if (c.path != KV_PATH_ZEROCOPY) continue;
         KvJob job;
-        fill_geometry(p, job);
+        fill_geometry(p, job, true);
         job.dir[0] = zerocopy_dir(p, c);
         job.dir[1] = KvDir{};
         job.dir[0].ctas = clamp_ctas(job, job.dir[0], p->dir[c.d].ctas);
-        KV_CUDA(p, launch_job(p, job, p->dir[c.d].stream));
+        KV_CUDA(p, launch_job(p, job, p->dir[c.d].stream, true));
     }
     // copy-engine directions, interleaved in slices so that both streams are fed from the start
     bool fin[2] = {true, true};
@@ -832,6 +839,8 @@ int32_t kv_pool_create(const kv_pool_config_t *cfg, kv_pool_t **out)
     }
     KV_CREATE_CUDA(cudaFuncSetAttribute(kv_copy_bulk<BULK_STAGE, BULK_NS, BULK_AHEAD>,
                                         cudaFuncAttributeMaxDynamicSharedMemorySize, BULK_STAGE * BULK_NS));
+    KV_CREATE_CUDA(cudaFuncSetAttribute(kv_copy_bulk<LINK_STAGE, LINK_NS, LINK_AHEAD>,
+                                        cudaFuncAttributeMaxDynamicSharedMemorySize, LINK_STAGE * LINK_NS));
 #undef KV_CREATE_CUDA
 
     try {

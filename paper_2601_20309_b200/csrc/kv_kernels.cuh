@@ -141,15 +141,21 @@ __device__ __forceinline__ unsigned long long kv_globaltimer()
     asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
     return t;
 }
-// bounded wait: gives up after about limit_ns
+// bounded wait: gives up after about limit_ns.  A short burst of polls catches HBM-latency waits;
+// after that the thread sleeps between polls, so a CTA that waits on the host link for microseconds
+// at a time does not take issue slots from whatever else runs on its SM.
 __device__ __forceinline__ bool kv_mbar_wait(uint32_t bar, uint32_t parity, unsigned long long limit_ns)
 {
-    if (kv_mbar_try_wait(bar, parity)) return true;
+#pragma unroll 1
+    for (int k = 0; k < 16; ++k)
+        if (kv_mbar_try_wait(bar, parity)) return true;
     const unsigned long long t0 = kv_globaltimer();
     for (;;) {
 #pragma unroll 1
-        for (int k = 0; k < 256; ++k)
+        for (int k = 0; k < 64; ++k) {
+            __nanosleep(200);
             if (kv_mbar_try_wait(bar, parity)) return true;
+        }
         if (kv_globaltimer() - t0 > limit_ns) return false;
     }
 }

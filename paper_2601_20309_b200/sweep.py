@@ -11,7 +11,13 @@
         contiguous or uniformly random, payload 64 MB .. G GB per direction, each direction alone
         and both at once, on every transfer path.  Its result is the table behind kv_path_for.
 
-Both print one JSON object per line and, at the end, a markdown table.
+    python -m paper_2601_20309_b200.sweep overlap [--out FILE]
+        Rotation beside compute (the paper's cross-iteration pipeline, section 4.3.2, hides transfers
+        behind model execution): a rotation of 2 GiB each way runs while a stand-in for a decode step
+        (back-to-back element-wise kernels over 1 GiB on a third stream: HBM-bound, every SM busy) runs too.  Reports
+        how much each slows the other, for the staged and the zero-copy path.
+
+All print one JSON object per line and, at the end, a markdown table.
 """
 from __future__ import annotations
 
@@ -126,9 +132,78 @@ def paths(out, max_payload_gb: float) -> None:
               f"{f('staged')} | {f('zerocopy')} | {f('ce2d')} | {f('naive')} | {f('auto')} | {r['auto_took']} |")
 
 
+def overlap(out) -> None:
+    import torch
+    shape = W.SHAPE_8B
+    n = 1024                                                   # 2 GiB each way
+    w = W.config4_sweep_case(16, False, n * shape.block_bytes, nb_host=16 * n)
+    rot = w.steps[0]
+    dev = torch.empty(w.nb_gpu * shape.block_bytes, dtype=torch.uint8, device="cuda:0")
+    src = torch.empty(1 << 30, dtype=torch.uint8, device="cuda:0")
+    dst = torch.empty_like(src)
+    side = torch.cuda.Stream()
+    pool = B.KVPool(shape.num_layers, shape.block_size, shape.kv_heads, shape.head_dim, w.nb_gpu, w.nb_host,
+                    dev.data_ptr())
+    nbytes = 2 * rot.n_out * shape.block_bytes
+
+    def compute(k):
+        """k stand-in decode steps on the side stream; returns (start, end) events."""
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        with torch.cuda.stream(side):
+            e0.record()
+            for _ in range(k):
+                torch.add(src, 1, out=dst)                     # an SM kernel (a plain copy could go to a copy engine)
+            e1.record()
+        return e0, e1
+
+    rows = []
+    for name, pid in (("staged", B.KV_PATH_STAGED), ("zerocopy", B.KV_PATH_ZEROCOPY)):
+        pool.kv_pool_set_path(pid, pid)
+        for _ in range(2):                                     # warm-up
+            pool.kv_rotate(rot.out_gpu, rot.out_host, rot.in_host, rot.in_gpu)
+            pool.kv_sync()
+        t_rot = []
+        for _ in range(3):
+            pool.kv_rotate(rot.out_gpu, rot.out_host, rot.in_host, rot.in_gpu)
+            pool.kv_sync()
+            t_rot.append(pool.kv_get_stats()["last_union_ms"])
+        rot_alone = min(t_rot)
+        alone = []
+        for _ in range(3):                                     # first round warms the kernel up
+            e0, e1 = compute(40)
+            torch.cuda.synchronize()
+            alone.append(e0.elapsed_time(e1) / 40)
+        step_alone = min(alone[1:])                            # ms per 1 GiB pass with nothing else running
+        k = max(4, int(1.3 * rot_alone / step_alone))          # compute outlasts the rotation a little
+        both_rot, both_step = [], []
+        for _ in range(3):
+            e0, e1 = compute(k)
+            pool.kv_rotate(rot.out_gpu, rot.out_host, rot.in_host, rot.in_gpu)
+            pool.kv_sync()
+            both_rot.append(pool.kv_get_stats()["last_union_ms"])
+            torch.cuda.synchronize()
+            both_step.append(e0.elapsed_time(e1) / k)
+        # the compute ran beside the rotation for rot/(k*step) of its time; scale its slowdown to that share
+        r_ms, s_ms = min(both_rot), min(both_step)
+        share = min(1.0, r_ms / (k * s_ms))
+        rec = {"path": name, "rotate_alone_gbs": round(nbytes / rot_alone / 1e6, 1), "rotate_beside_compute_gbs": round(nbytes / r_ms / 1e6, 1),
+               "compute_alone_tbs": round(2 * (1 << 30) / step_alone / 1e9, 2), "compute_beside_rotate_tbs": round(2 * (1 << 30) / s_ms / 1e9, 2),
+               "compute_slowdown_pct_over_whole_run": round(100 * (s_ms / step_alone - 1), 2),
+               "compute_slowdown_pct_while_rotating": round(100 * (s_ms / step_alone - 1) / share, 2),
+               "rotate_slowdown_pct": round(100 * (r_ms / rot_alone - 1), 2), "decode_steps": k}
+        rows.append(rec)
+        _emit(rec, out)
+    pool.destroy()
+    print("\n| path | rotate alone GB/s | rotate beside compute GB/s | compute alone TB/s | compute beside rotate TB/s | "
+          "compute slowdown while rotating | rotate slowdown |\n|---|---|---|---|---|---|---|")
+    for r in rows:
+        print(f"| {r['path']} | {r['rotate_alone_gbs']} | {r['rotate_beside_compute_gbs']} | {r['compute_alone_tbs']} | "
+              f"{r['compute_beside_rotate_tbs']} | {r['compute_slowdown_pct_while_rotating']} % | {r['rotate_slowdown_pct']} % |")
+
+
 def main() -> None:
     ap = argparse.ArgumentParser()
-    ap.add_argument("what", choices=["probe", "paths"])
+    ap.add_argument("what", choices=["probe", "paths", "overlap"])
     ap.add_argument("--out", default=None)
     ap.add_argument("--max-payload-gb", type=float, default=4.0)
     a = ap.parse_args()
@@ -138,8 +213,10 @@ def main() -> None:
     out = open(a.out, "w") if a.out else None
     if a.what == "probe":
         probe(out)
-    else:
+    elif a.what == "paths":
         paths(out, a.max_payload_gb)
+    else:
+        overlap(out)
 
 
 if __name__ == "__main__":
