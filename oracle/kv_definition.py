@@ -71,11 +71,15 @@ class KVDefinition:
     """Both pools as 6-D ``uint16`` arrays; every move is one indexed assignment."""
 
     def __init__(self, num_layers, block_size, kv_heads, head_dim,
-                 num_gpu_blocks, num_host_blocks, host_layout=BLOCK_FIRST):
+                 num_gpu_blocks, num_host_blocks, host_layout=BLOCK_FIRST, dev_layout=LAYER_FIRST):
         self.L, self.bs, self.H, self.D = num_layers, block_size, kv_heads, head_dim
         self.nb_gpu, self.nb_host = num_gpu_blocks, num_host_blocks
         self.host_layout = host_layout
-        self.G = np.zeros((num_layers, 2, num_gpu_blocks, block_size, kv_heads, head_dim), np.uint16)
+        self.dev_layout = dev_layout
+        if dev_layout == LAYER_FIRST:
+            self.G = np.zeros((num_layers, 2, num_gpu_blocks, block_size, kv_heads, head_dim), np.uint16)
+        else:       # the paper's block-first storage order, applied to the device pool
+            self.G = np.zeros((num_gpu_blocks, num_layers, 2, block_size, kv_heads, head_dim), np.uint16)
         if host_layout == BLOCK_FIRST:
             self.Hs = np.zeros((num_host_blocks, num_layers, 2, block_size, kv_heads, head_dim), np.uint16)
         else:
@@ -83,14 +87,14 @@ class KVDefinition:
 
     # logical accessors: the (block_size, kv_heads, head_dim) words of one plane of one block
     def g_seg(self, l, kv, b):
-        return self.G[l, kv, b]
+        return self.G[l, kv, b] if self.dev_layout == LAYER_FIRST else self.G[b, l, kv]
 
     def h_seg(self, l, kv, h):
         return self.Hs[h, l, kv] if self.host_layout == BLOCK_FIRST else self.Hs[l, kv, h]
 
     def g_block(self, b):
         """All 2L planes of device block b, shape (L, 2, bs, H, D)."""
-        return self.G[:, :, b]
+        return self.G[:, :, b] if self.dev_layout == LAYER_FIRST else self.G[b]
 
     def h_block(self, h):
         return self.Hs[h] if self.host_layout == BLOCK_FIRST else self.Hs[:, :, h]

@@ -40,7 +40,7 @@ typedef struct {
     int64_t num_gpu_blocks;
     int64_t num_host_blocks;
     int32_t host_layout; /* 0 = block-first, 1 = layer-first */
-    int32_t pad_;
+    int32_t dev_layout;  /* 0 = layer-first, 1 = block-first (the paper's redesigned storage order) */
 } kvo_shape_t;
 
 enum {
@@ -63,10 +63,14 @@ int64_t kvo_blk_bytes(const kvo_shape_t *s)
     return 2 * (int64_t)s->num_layers * kvo_seg_bytes(s);
 }
 
-/* layer-first: inside one (layer, plane) consecutive blocks are SEG apart */
+/* layer-first: inside one (layer, plane) consecutive blocks are SEG apart;
+ * block-first: all planes of a block are contiguous and consecutive blocks are one whole block apart
+ * (section 4.3.2: the stride between block i and block j grows from (j-i)*S_seg to (j-i)*N_L*S_seg) */
 int64_t kvo_dev_off(const kvo_shape_t *s, int64_t l, int64_t kv, int64_t b)
 {
     int64_t plane = l * 2 + kv;
+    if (s->dev_layout == 1)
+        return b * kvo_blk_bytes(s) + plane * kvo_seg_bytes(s);
     return (plane * s->num_gpu_blocks + b) * kvo_seg_bytes(s);
 }
 

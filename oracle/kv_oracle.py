@@ -24,7 +24,7 @@ class _Shape(C.Structure):
     _fields_ = [("num_layers", C.c_int32), ("block_size", C.c_int32),
                 ("kv_heads", C.c_int32), ("head_dim", C.c_int32),
                 ("num_gpu_blocks", C.c_int64), ("num_host_blocks", C.c_int64),
-                ("host_layout", C.c_int32), ("pad_", C.c_int32)]
+                ("host_layout", C.c_int32), ("dev_layout", C.c_int32)]
 
 
 _lib = None
@@ -63,9 +63,9 @@ def _ids(a):
 
 class ByteOracle:
     def __init__(self, num_layers, block_size, kv_heads, head_dim,
-                 num_gpu_blocks, num_host_blocks, host_layout=0, alloc=True):
+                 num_gpu_blocks, num_host_blocks, host_layout=0, alloc=True, dev_layout=0):
         self.shape = _Shape(num_layers, block_size, kv_heads, head_dim,
-                            num_gpu_blocks, num_host_blocks, host_layout, 0)
+                            num_gpu_blocks, num_host_blocks, host_layout, dev_layout)
         self.seg = lib().kvo_seg_bytes(C.byref(self.shape))
         self.blk = lib().kvo_blk_bytes(C.byref(self.shape))
         if alloc:

@@ -389,3 +389,48 @@ def test_planted_mistakes_are_caught():
     bad.G[...], bad.Hs[...] = G0, H0
     bad.rotate([2], [1], [1], [0], allow_overlap=True)
     assert not np.array_equal(bad.G[:, :, 0], G0[:, :, 2])                  # sequential-semantics pin fails
+
+
+# ------------------------------------------------------------ block-first DEVICE layout (the paper's redesign)
+
+def test_block_first_device_layout_strides_and_paper_sizes():
+    """Section 4.3.2: with block-first storage all layers of a block are contiguous (64 KB segments merge
+    into one 4 MB region for Qwen2.5-32B) and the stride between blocks i and j is (j-i)*N_L*S_seg."""
+    g = read_golden("paper_sizes.txt")
+    L, bs, H, Dm = g["num_layers"], g["block_size"], g["kv_heads"], g["head_dim"]
+    c = ByteOracle(L, bs, H, Dm, 9, 9, alloc=False, dev_layout=1)
+    assert c.dev_off(0, 0, 1) - c.dev_off(0, 0, 0) == g["block_bytes"] == L * g["segment_bytes_k_plus_v"]
+    assert c.dev_off(1, 0, 0) - c.dev_off(0, 0, 0) == g["segment_bytes_k_plus_v"]      # next layer: next segment
+    assert c.dev_off(0, 1, 0) - c.dev_off(0, 0, 0) == g["segment_bytes_k_plus_v"] // 2  # V plane follows K plane
+    small = ByteOracle(5, 4, 2, 8, 11, 13, alloc=False, dev_layout=1)
+    seg = small.seg
+    for l, kv, i, j in itertools.product(range(5), range(2), (0, 3), (1, 10)):
+        assert small.dev_off(l, kv, j) - small.dev_off(l, kv, i) == (j - i) * 5 * (2 * seg)
+    offs = sorted(small.dev_off(l, kv, b) for l in range(5) for kv in range(2) for b in range(11))
+    assert offs == list(range(0, 2 * 5 * 11 * seg, seg))
+    # the same rule as the block-first host pool
+    assert all(small.dev_off(l, kv, b) == small.host_off(b, l, kv) for l in range(5) for kv in range(2) for b in range(11))
+
+
+@pytest.mark.parametrize("host_layout", [D.BLOCK_FIRST, D.LAYER_FIRST])
+def test_block_first_device_layout_moves_the_same_logical_content(host_layout):
+    """Changing where the device pool keeps a plane must not change what a rotation does to the logical
+    content: byte oracle and 6-D definition, both on the block-first device layout, against the
+    layer-first pair on the same logical data and lists."""
+    rng = np.random.default_rng(21)
+    L, bs, H, Dm, nbg, nbh = 3, 4, 2, 8, 10, 12
+    dl = D.KVDefinition(L, bs, H, Dm, nbg, nbh, host_layout)                       # layer-first device
+    db = D.KVDefinition(L, bs, H, Dm, nbg, nbh, host_layout, dev_layout=D.BLOCK_FIRST)
+    cb = ByteOracle(L, bs, H, Dm, nbg, nbh, host_layout, dev_layout=1)
+    dl.G[...] = rng.integers(0, 65536, dl.G.shape, dtype=np.uint16)
+    dl.Hs[...] = rng.integers(0, 65536, dl.Hs.shape, dtype=np.uint16)
+    db.G[...] = np.moveaxis(dl.G, 2, 0)                                             # same logical content
+    db.Hs[...] = dl.Hs
+    cb.G[:] = db.G.reshape(-1).view(np.uint8)                                       # row-major = the byte layout
+    cb.Hs[:] = db.Hs.reshape(-1).view(np.uint8)
+    for _ in range(5):
+        og, oh, ih, ig = random_lists(rng, nbg, nbh, 4, 3)
+        assert dl.rotate(og, oh, ih, ig) == db.rotate(og, oh, ih, ig) == cb.rotate(og, oh, ih, ig) == 0
+    assert np.array_equal(np.moveaxis(dl.G, 2, 0), db.G) and np.array_equal(dl.Hs, db.Hs)
+    assert np.array_equal(cb.G.view(np.uint16), db.G.reshape(-1))
+    assert np.array_equal(cb.Hs.view(np.uint16), db.Hs.reshape(-1))
