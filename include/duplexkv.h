@@ -9,7 +9,8 @@
  * that the host link is used full-duplex.
  *
  * Layouts (elements are 16-bit words, never interpreted):
- *   device pool   [layer][K|V][block][block_size][kv_heads][head_dim]      ("layer-first")
+ *   device pool   [layer][K|V][block][block_size][kv_heads][head_dim]      ("layer-first", default), or
+ *                 block-first like the host pool (KV_DEV_BLOCK_FIRST)
  *   host pool     [block][layer][K|V][block_size][kv_heads][head_dim]      ("block-first", default;
  *                 the paper's merged layout: all layers of one block contiguous), or layer-first
  *                 like the device pool.
@@ -51,6 +52,10 @@ extern "C" {
 /* host pool layout */
 #define KV_HOST_BLOCK_FIRST   0
 #define KV_HOST_LAYER_FIRST   1
+
+/* device pool layout */
+#define KV_DEV_LAYER_FIRST    0     /* [layer][K|V][block]...: the layout the engine is built for        */
+#define KV_DEV_BLOCK_FIRST    1     /* [block][layer][K|V]...: the paper's redesigned storage order      */
 
 /* transfer paths (how the host link is driven) */
 #define KV_PATH_AUTO          0     /* per call: STAGED when the copy-engine transfers the call needs would
@@ -96,6 +101,11 @@ typedef struct {
     int32_t path_in;        /* KV_PATH_* of the swap-in direction; KV_PATH_AUTO (0) = same as `path`      */
     int32_t ce_streams;     /* streams per direction that the copy-engine paths spread their transfers
                                over (1..4), 0 = 1                                                         */
+    int32_t device_layout;  /* KV_DEV_LAYER_FIRST (default) or KV_DEV_BLOCK_FIRST: the variant of section
+                               4.3.2 in which all layers of a device block are contiguous (a consumer of
+                               the pool then strides by BLK between blocks).  kv_gather_blocks_static
+                               reads layer-first pools only                                               */
+    int32_t pad_;
 } kv_pool_config_t;
 
 typedef struct {

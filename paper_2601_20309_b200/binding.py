@@ -27,6 +27,9 @@ KV_ERR_UNSUPPORTED = -8
 KV_HOST_BLOCK_FIRST = 0
 KV_HOST_LAYER_FIRST = 1
 
+KV_DEV_LAYER_FIRST = 0
+KV_DEV_BLOCK_FIRST = 1
+
 KV_PATH_AUTO = 0
 KV_PATH_ZEROCOPY = 1
 KV_PATH_STAGED = 2
@@ -46,7 +49,8 @@ class kv_pool_config_t(C.Structure):
                 ("device_base", C.c_void_p), ("host_base", C.c_void_p), ("host_layout", C.c_int32),
                 ("device_id", C.c_int32), ("stream_out", C.c_void_p), ("stream_in", C.c_void_p),
                 ("path", C.c_int32), ("flags", C.c_int32), ("ctas_out", C.c_int32), ("ctas_in", C.c_int32),
-                ("staging_bytes", C.c_int64), ("path_in", C.c_int32), ("ce_streams", C.c_int32)]
+                ("staging_bytes", C.c_int64), ("path_in", C.c_int32), ("ce_streams", C.c_int32),
+                ("device_layout", C.c_int32), ("pad_", C.c_int32)]
 
 
 class kv_stats_t(C.Structure):
@@ -248,11 +252,12 @@ class KVPool:
                  host_base: Optional[int] = None, host_layout: int = KV_HOST_BLOCK_FIRST,
                  device_id: int = 0, stream_out: Optional[int] = None, stream_in: Optional[int] = None,
                  path: int = KV_PATH_AUTO, flags: int = 0, ctas_out: int = 0, ctas_in: int = 0,
-                 staging_bytes: int = 0, path_in: int = KV_PATH_AUTO, ce_streams: int = 0):
+                 staging_bytes: int = 0, path_in: int = KV_PATH_AUTO, ce_streams: int = 0,
+                 device_layout: int = KV_DEV_LAYER_FIRST):
         self.cfg = kv_pool_config_t(num_layers, block_size, kv_heads, head_dim, num_gpu_blocks,
                                     num_host_blocks, device_base, host_base, host_layout, device_id,
                                     stream_out, stream_in, path, flags, ctas_out, ctas_in, staging_bytes,
-                                    path_in, ce_streams)
+                                    path_in, ce_streams, device_layout, 0)
         self._h = C.c_void_p()
         rc = lib().kv_pool_create(C.byref(self.cfg), C.byref(self._h))
         if rc != KV_OK:

@@ -130,9 +130,22 @@ int32_t fail_cuda(kv_pool *p, cudaError_t e, const char *what)
         if (e_ != cudaSuccess) return fail_cuda((p), e_, #expr);  \
     } while (0)
 
+bool dev_block_first(const kv_pool *p) { return p->cfg.device_layout == KV_DEV_BLOCK_FIRST; }
+
 KvSide device_side(const kv_pool *p)
 {
+    if (dev_block_first(p)) return KvSide{(unsigned long long)p->dev, p->blk, p->seg};
     return KvSide{(unsigned long long)p->dev, p->seg, p->cfg.num_gpu_blocks * p->seg};
+}
+
+// device address of the first plane of block g, and the distance between its planes
+inline uint8_t *dev_block_ptr(const kv_pool *p, int32_t g)
+{
+    return p->dev + (int64_t)g * (dev_block_first(p) ? p->blk : p->seg);
+}
+inline size_t dev_pitch(const kv_pool *p)
+{
+    return (size_t)(dev_block_first(p) ? p->seg : p->cfg.num_gpu_blocks * p->seg);
 }
 
 KvSide host_side(const kv_pool *p)
@@ -498,7 +511,7 @@ int32_t ce_issue_some(kv_pool *p, DirCall &c, int budget, bool &finished)
         const int64_t total = c.n * p->planes;
         while (budget-- > 0 && c.ce_next < total) {
             const int64_t i = c.ce_next / p->planes, pl = c.ce_next % p->planes;
-            uint8_t *dv = p->dev + (pl * p->cfg.num_gpu_blocks + c.gpu_ids[i]) * p->seg;
+            uint8_t *dv = dev_block_ptr(p, c.gpu_ids[i]) + pl * (int64_t)dev_pitch(p);
             uint8_t *hv = host_block_ptr(p, c.host_ids[i]) + pl * (int64_t)host_pitch(p);
             KV_CUDA(p, cudaMemcpyAsync(c.d == 0 ? hv : dv, c.d == 0 ? dv : hv, (size_t)p->seg, kind, s.sub[i % s.nsub]));
             p->stats.ce_copies++;
@@ -508,14 +521,17 @@ int32_t ce_issue_some(kv_pool *p, DirCall &c, int budget, bool &finished)
         return KV_OK;
     }
     if (c.path == KV_PATH_CE2D) {
-        // one strided transfer per block: `planes` rows of SEG bytes
+        // one transfer per block: `planes` rows of SEG bytes, strided where a pool is layer-first; a
+        // plain BLK-byte transfer when both pools are block-first (the paper's one-copy-per-merged-region)
         while (budget-- > 0 && c.ce_next < c.n) {
             const int64_t i = c.ce_next;
-            uint8_t *dv = p->dev + (int64_t)c.gpu_ids[i] * p->seg;
+            uint8_t *dv = dev_block_ptr(p, c.gpu_ids[i]);
             uint8_t *hv = host_block_ptr(p, c.host_ids[i]);
-            const size_t dpitch = (size_t)(p->cfg.num_gpu_blocks * p->seg);
+            const size_t dpitch = dev_pitch(p);
             cudaStream_t cs = s.sub[i % s.nsub];
-            if (c.d == 0)
+            if (dpitch == (size_t)p->seg && host_pitch(p) == (size_t)p->seg)
+                KV_CUDA(p, cudaMemcpyAsync(c.d == 0 ? hv : dv, c.d == 0 ? dv : hv, (size_t)p->blk, kind, cs));
+            else if (c.d == 0)
                 KV_CUDA(p, cudaMemcpy2DAsync(hv, host_pitch(p), dv, dpitch, (size_t)p->seg, (size_t)p->planes, kind, cs));
             else
                 KV_CUDA(p, cudaMemcpy2DAsync(dv, dpitch, hv, host_pitch(p), (size_t)p->seg, (size_t)p->planes, kind, cs));
@@ -740,6 +756,8 @@ int32_t kv_pool_create(const kv_pool_config_t *cfg, kv_pool_t **out)
         return fail(nullptr, KV_ERR_INVALID_ARG, "host_base must be 4096-byte aligned");
     if (cfg->host_layout != KV_HOST_BLOCK_FIRST && cfg->host_layout != KV_HOST_LAYER_FIRST)
         return fail(nullptr, KV_ERR_INVALID_ARG, "unknown host_layout");
+    if (cfg->device_layout != KV_DEV_LAYER_FIRST && cfg->device_layout != KV_DEV_BLOCK_FIRST)
+        return fail(nullptr, KV_ERR_INVALID_ARG, "unknown device_layout");
     if (cfg->path < KV_PATH_AUTO || cfg->path > KV_PATH_NAIVE || cfg->path_in < KV_PATH_AUTO || cfg->path_in > KV_PATH_NAIVE)
         return fail(nullptr, KV_ERR_INVALID_ARG, "unknown path");
     if (cfg->ctas_out < 0 || cfg->ctas_in < 0 || cfg->staging_bytes < 0 || cfg->ce_streams < 0 ||

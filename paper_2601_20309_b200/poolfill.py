@@ -36,8 +36,10 @@ class Layout:
         self.base, self.blk_stride, self.plane_stride, self.shape = base, blk_stride, plane_stride, shape
 
     @staticmethod
-    def device(base: int, shape: W.KVShape, num_blocks: int) -> "Layout":
+    def device(base: int, shape: W.KVShape, num_blocks: int, block_first: bool = False) -> "Layout":
         seg = 2 * shape.words_per_plane
+        if block_first:
+            return Layout(base, shape.block_bytes, seg, shape)
         return Layout(base, seg, num_blocks * seg, shape)
 
     @staticmethod

@@ -76,7 +76,7 @@ PATHS = [("staged", B.KV_PATH_STAGED), ("zerocopy", B.KV_PATH_ZEROCOPY), ("ce2d"
          ("naive", B.KV_PATH_NAIVE), ("auto", B.KV_PATH_AUTO)]
 
 
-def paths(out, max_payload_gb: float) -> None:
+def paths(out, max_payload_gb: float, device_layout: int = 0) -> None:
     import torch
     rows = []
     payloads = [p for p in (64e6, 256e6, 1e9, 4e9, 8e9) if p <= max_payload_gb * 1e9 + 1]
@@ -92,7 +92,7 @@ def paths(out, max_payload_gb: float) -> None:
                 dev = torch.empty(w.nb_gpu * shape.block_bytes, dtype=torch.uint8, device="cuda:0")
                 probe_bi = B.kv_probe_link(0, 256 * M, 2)["bi_sum_gbs"]
                 pool = B.KVPool(shape.num_layers, shape.block_size, shape.kv_heads, shape.head_dim, w.nb_gpu,
-                                w.nb_host, dev.data_ptr())
+                                w.nb_host, dev.data_ptr(), device_layout=device_layout)
                 nbytes = rot.n_out * shape.block_bytes
 
                 def best(fn, reps):
@@ -206,6 +206,8 @@ def main() -> None:
     ap.add_argument("what", choices=["probe", "paths", "overlap"])
     ap.add_argument("--out", default=None)
     ap.add_argument("--max-payload-gb", type=float, default=4.0)
+    ap.add_argument("--device-layout", choices=["layer-first", "block-first"], default="layer-first",
+                    help="paths: device pool layout (block-first = the paper's redesigned storage order)")
     a = ap.parse_args()
     import torch
     if not torch.cuda.is_available():
@@ -214,7 +216,7 @@ def main() -> None:
     if a.what == "probe":
         probe(out)
     elif a.what == "paths":
-        paths(out, a.max_payload_gb)
+        paths(out, a.max_payload_gb, 1 if a.device_layout == "block-first" else 0)
     else:
         overlap(out)
 

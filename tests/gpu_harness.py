@@ -10,12 +10,13 @@ from paper_2601_20309_b200 import workload as W
 class Pair:
     """A GPU pool (through the C ABI) and the byte oracle holding the same logical content."""
 
-    def __init__(self, shape, nb_gpu, nb_host, seed=1, host_layout=0, **pool_kw):
+    def __init__(self, shape, nb_gpu, nb_host, seed=1, host_layout=0, device_layout=0, **pool_kw):
         import torch
         self.torch = torch
         self.shape, self.nb_gpu, self.nb_host, self.seed = shape, nb_gpu, nb_host, seed
         s = shape
-        self.oracle = ByteOracle(s.num_layers, s.block_size, s.kv_heads, s.head_dim, nb_gpu, nb_host, host_layout)
+        self.oracle = ByteOracle(s.num_layers, s.block_size, s.kv_heads, s.head_dim, nb_gpu, nb_host, host_layout,
+                                 dev_layout=device_layout)
         o = self.oracle
         wpp = s.words_per_plane
         G16 = o.G.view(np.uint16)
@@ -32,7 +33,7 @@ class Pair:
                 H16[off:off + wpp] = words[pl]
         self.dev = torch.from_numpy(o.G.copy()).to("cuda:0")
         self.pool = B.KVPool(s.num_layers, s.block_size, s.kv_heads, s.head_dim, nb_gpu, nb_host,
-                             self.dev.data_ptr(), host_layout=host_layout, **pool_kw)
+                             self.dev.data_ptr(), host_layout=host_layout, device_layout=device_layout, **pool_kw)
         self.pool.host_array()[:] = o.Hs
 
     def gpu_bytes(self):

@@ -341,3 +341,30 @@ def test_rotate_swap_in_waits_for_an_earlier_swap_out_that_reads_its_destination
         p.assert_equal("rotate behind a long swap-out")
     finally:
         p.close()
+
+
+@pytest.mark.parametrize("path", list(PATHS))
+@pytest.mark.parametrize("host_layout", [0, 1], ids=["hostblockfirst", "hostlayerfirst"])
+def test_block_first_device_layout(path, host_layout):
+    """The paper's redesigned storage order applied to the device pool: all planes of a block contiguous.
+    Same calls, same oracle results through the logical accessor; on the copy-engine path with a
+    block-first host pool a block is then one plain transfer."""
+    w = W.config1_tiny()
+    p = _pair(w.shape, w.nb_gpu, w.nb_host, seed=w.seed, host_layout=host_layout, device_layout=1, path=PATHS[path])
+    try:
+        assert p.rotate_both(w.steps[0]) == 0
+        p.assert_equal(f"block-first device, {path}")
+        st = p.pool.kv_get_stats()
+        if path == "ce2d":
+            assert st["ce_copies"] == w.steps[0].n_out + w.steps[0].n_in
+    finally:
+        p.close()
+    w = W.config2_8b(nb_gpu=320, nb_host=448, n_req=16, median=96, max_tokens=512, n_rot=4)
+    p = _pair(w.shape, w.nb_gpu, w.nb_host, seed=w.seed, host_layout=host_layout, device_layout=1, path=PATHS[path])
+    try:
+        assert p.rotate_both(w.steps[0]) == 0
+        for r in w.extra["pairs"][:3]:
+            assert p.rotate_both(r) == 0
+        p.assert_equal(f"block-first device 8B shape, {path}")
+    finally:
+        p.close()
