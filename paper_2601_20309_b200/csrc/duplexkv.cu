@@ -357,9 +357,13 @@ int32_t plan_staged(kv_pool *p, DirCall &c)
         // The first chunk of a swap-out is half as long as the rest: its first transfer starts sooner, and
         // in a rotation the pack kernels then run midway between the swap-in's unpack kernels instead of
         // at the same moments (both directions advance one chunk per equal stretch of link time).
-        const int64_t first = (c.d == 0 && c.n > s.half_blocks) ? std::max<int64_t>(1, s.half_blocks / 2) : s.half_blocks;
+        // A call that would fit one half is still cut into about four chunks (of 8 MiB or more), so that its
+        // own packing, transfers and unpacking overlap instead of following one another.
+        const int64_t min_chunk = std::max<int64_t>(1, (8ll << 20) / p->blk);
+        const int64_t chunk = std::min(s.half_blocks, std::max(min_chunk, (c.n + 3) / 4));
+        const int64_t first = (c.d == 0 && c.n > chunk) ? std::max<int64_t>(1, chunk / 2) : chunk;
         for (int64_t lo = 0, hi = 0; lo < c.n; lo = hi) {
-            hi = std::min(c.n, lo + (lo == 0 ? first : s.half_blocks));
+            hi = std::min(c.n, lo + (lo == 0 ? first : chunk));
             CeChunk ch{lo, hi, (int32_t)s.ops.size(), 0};
             if (layer_first) {
                 // one strided transfer per block: `planes` rows of SEG bytes, a whole host plane apart
