@@ -276,6 +276,15 @@ typedef struct {
 } kv_pool_shape_t;
 int32_t kv_pool_shape(kv_pool_t *pool, kv_pool_shape_t *out);
 
+/*
+ * Make `stream` (a cudaStream_t of the pool's device; NULL = the default stream) wait, on the device and
+ * without blocking the host, for everything issued so far in the given directions (bit 0 = swap-outs,
+ * bit 1 = swap-ins; 3 = both).  This is how a compute stream picks up swapped-in blocks, or holds back
+ * writes to blocks a swap-out still reads, in the paper's cross-iteration pipeline (section 4.3.2), where
+ * rotation runs beside model execution and nobody wants a host-side kv_sync.
+ */
+int32_t kv_stream_wait(kv_pool_t *pool, void *stream, int32_t directions);
+
 /* Calls issued and calls known to have completed, per direction (a non-blocking look at the pool's
  * end events).  Any pointer may be NULL.  kv_gather_blocks / kv_scatter_blocks count as calls of the
  * out / in direction. */

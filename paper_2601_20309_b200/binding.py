@@ -95,7 +95,7 @@ class kv_table_stats_t(C.Structure):
 EXPORTS = ["kv_pool_create", "kv_pool_destroy", "kv_pool_set_path", "kv_swap_out", "kv_swap_in", "kv_rotate", "kv_sync",
            "kv_gather_blocks", "kv_scatter_blocks", "kv_host_ptr", "kv_get_stats", "kv_last_error",
            "kv_seg_bytes", "kv_blk_bytes", "kv_path_for", "kv_probe_link", "kv_probe_link_ex",
-           "kv_gather_blocks_static", "kv_pool_shape", "kv_pool_progress",
+           "kv_gather_blocks_static", "kv_pool_shape", "kv_pool_progress", "kv_stream_wait",
            "kv_table_create", "kv_table_create_dry", "kv_table_destroy", "kv_table_last_error", "kv_req_add",
            "kv_req_append", "kv_eager_rotate", "kv_req_rotate", "kv_req_preempt", "kv_req_resume", "kv_req_finish",
            "kv_req_info", "kv_req_blocks", "kv_table_get_stats"]
@@ -146,6 +146,8 @@ def lib() -> C.CDLL:
     i64p = C.POINTER(C.c_int64)
     L.kv_pool_shape.restype = C.c_int32
     L.kv_pool_shape.argtypes = [vp, C.POINTER(kv_pool_shape_t)]
+    L.kv_stream_wait.restype = C.c_int32
+    L.kv_stream_wait.argtypes = [vp, vp, C.c_int32]
     L.kv_pool_progress.restype = C.c_int32
     L.kv_pool_progress.argtypes = [vp, i64p, i64p, i64p, i64p]
     L.kv_table_create.restype = C.c_int32
@@ -342,6 +344,9 @@ class KVPool:
 
     def kv_last_error(self) -> str:
         return lib().kv_last_error(self._h).decode()
+
+    def kv_stream_wait(self, stream: Optional[int], directions: int = 3, check: bool = True) -> int:
+        return self._ret(lib().kv_stream_wait(self._h, stream, directions), check)
 
     def kv_pool_progress(self) -> dict:
         v = [C.c_int64() for _ in range(4)]

@@ -1150,6 +1150,17 @@ int32_t kv_scatter_blocks(kv_pool_t *p, const void *src_device, const int32_t *g
     return device_leg(p, gpu_ids, n, src_device, 1);
 }
 
+int32_t kv_stream_wait(kv_pool_t *p, void *stream, int32_t directions)
+{
+    if (!p || (directions & ~3) || directions == 0) return KV_ERR_INVALID_ARG;
+    for (int d = 0; d < 2; ++d) {
+        DirState &s = p->dir[d];
+        if (!(directions & (1 << d)) || s.issued == 0) continue;
+        KV_CUDA(p, cudaStreamWaitEvent((cudaStream_t)stream, s.ev_end[s.issued % KV_SLOTS], 0));
+    }
+    return KV_OK;
+}
+
 int32_t kv_pool_progress(kv_pool_t *p, int64_t *out_issued, int64_t *out_done, int64_t *in_issued, int64_t *in_done)
 {
     if (!p) return KV_ERR_INVALID_ARG;

@@ -368,3 +368,28 @@ def test_block_first_device_layout(path, host_layout):
         p.assert_equal(f"block-first device 8B shape, {path}")
     finally:
         p.close()
+
+
+def test_stream_wait_orders_a_consumer_stream_behind_the_swap_in():
+    """No host-side sync: a torch stream that was told to wait for the pool reads swapped-in blocks only
+    after they have landed."""
+    import torch
+    shape = W.KVShape(32, 16, 8, 128)                 # 2 MiB blocks
+    nbg, nbh = 260, 300
+    p = _pair(shape, nbg, nbh, seed=21, path=PATHS["zerocopy"])
+    try:
+        ih = np.arange(0, 250, dtype=np.int32)
+        ig = np.arange(0, 250, dtype=np.int32)        # 500 MiB over the link: about 10 ms
+        assert p.oracle.swap_in(ih, ig) == 0
+        snap = torch.empty_like(p.dev)
+        consumer = torch.cuda.Stream()
+        assert p.pool.kv_swap_in(ih, ig) == 0
+        assert p.pool.kv_stream_wait(consumer.cuda_stream, 2) == 0
+        with torch.cuda.stream(consumer):
+            snap.copy_(p.dev, non_blocking=True)      # would see half-written blocks without the wait
+        consumer.synchronize()
+        assert np.array_equal(snap.cpu().numpy(), p.oracle.G)
+        assert p.pool.kv_stream_wait(None, 0, check=False) == -1
+        p.assert_equal("after stream wait")
+    finally:
+        p.close()

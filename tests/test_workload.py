@@ -1,4 +1,4 @@
-"""Seeded input generators: determinism, the shapes BASELINE's five workloads ask for, and the
+"""Seeded input generators: determinism, the shapes of the five workloads, and the
 block-table bookkeeping (one residency per request, table length, pool-wide unique ids)."""
 import numpy as np
 import pytest
