@@ -37,6 +37,8 @@ from paper_2601_20309_b200 import workload as W         # noqa: E402
 
 METRIC = "full-duplex KV swap GB/s (out+in)"
 UNIT = "GB/s"
+WORKLOAD = ("config2 llama-3-8b-shaped KV (32 layers, 8 kv heads, head_dim 128, block 16, bf16): "
+            "paired rotate of %d requests each way per step")
 # DRAM traffic of one pack / unpack launch, from the ncu capture of an 89-block (186.65 MB) launch on the
 # --small case: dram__bytes_read.sum = 1.00005 x payload (no byte read twice); dram__bytes_write.sum =
 # payload - 48.5 MB, the lines still in L2 when the kernel ends.  Reads scale with the payload, the L2
@@ -166,7 +168,7 @@ def run_reference(args, rank: int) -> None:
     line = {"impl": "reference", "metric": METRIC, "value": val, "unit": UNIT, "n_gpus": args.gpus,
             "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms, "higher_is_better": True,
             "scaling": "weak", "vs_baseline": None, "dtype": "u16", "data": "synthetic",
-            "config": {"workload": "config2 llama-3-8b-shaped KV, paired rotate 16 requests each way (CPU sample)"},
+            "config": {"workload": WORKLOAD % 16, "cpu_sample": sample},
             "cpu_baseline": {"value": val, "unit": UNIT, "cores": threads, "kind": "oracle", "sample": sample},
             "e2e": {"value": val, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
             "gpu_launches": 0}
@@ -411,8 +413,7 @@ def run_ours(args, rank: int, local_rank: int, world: int) -> None:
             "warmup": args.warmup, "ms_per_step": step_ms, "higher_is_better": True, "scaling": "weak",
             "vs_baseline": None, "dtype": "u16", "data": "synthetic",
             "config": {"workload": ("SMALL profiling case of " if args.small else "") +
-                                   "config2 llama-3-8b-shaped KV (32 layers, 8 kv heads, head_dim 128, block 16, bf16): "
-                                   "paired rotate of %d requests each way per step" % (len(rot.out_req_offsets) - 1),
+                                   WORKLOAD % (len(rot.out_req_offsets) - 1),
                        "gpu_pool_blocks": nb_gpu, "host_pool_blocks": nb_host, "host_pool_shrunk": shrunk,
                        "blocks_out": int(rot.n_out), "blocks_in": int(rot.n_in), "block_bytes": shape.block_bytes,
                        "bytes_out_per_step": bytes_out, "bytes_in_per_step": bytes_in,
