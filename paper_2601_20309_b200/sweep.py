@@ -17,6 +17,11 @@
         (back-to-back element-wise kernels over 1 GiB on a third stream: HBM-bound, every SM busy) runs too.  Reports
         how much each slows the other, for the staged and the zero-copy path.
 
+    python -m paper_2601_20309_b200.sweep latency [--out FILE]
+        Call-to-completion time of small rotations (1 .. 256 blocks each way, 8B shape, scattered ids):
+        host clock around kv_rotate + kv_sync, median of 40, per path.  What a per-request rotate costs
+        when the link is not the limit.
+
 All print one JSON object per line and, at the end, a markdown table.
 """
 from __future__ import annotations
@@ -201,9 +206,45 @@ def overlap(out) -> None:
               f"{r['compute_beside_rotate_tbs']} | {r['compute_slowdown_pct_while_rotating']} % | {r['rotate_slowdown_pct']} % |")
 
 
+def latency(out) -> None:
+    import time
+    import numpy as np
+    import torch
+    shape = W.SHAPE_8B
+    nb = 4096
+    dev = torch.empty(nb * shape.block_bytes, dtype=torch.uint8, device="cuda:0")
+    pool = B.KVPool(shape.num_layers, shape.block_size, shape.kv_heads, shape.head_dim, nb, nb, dev.data_ptr())
+    rng = np.random.default_rng(3)
+    rows = []
+    for n in (1, 2, 4, 8, 16, 64, 256):
+        pg, ph = rng.permutation(nb).astype(np.int32), rng.permutation(nb).astype(np.int32)
+        og, ig, oh, ih = pg[:n], pg[n:2 * n], ph[:n], ph[n:2 * n]
+        rec = {"blocks_each_way": n, "mib_each_way": n * shape.block_bytes / M}
+        for name, pid in (("auto", B.KV_PATH_AUTO), ("staged", B.KV_PATH_STAGED), ("zerocopy", B.KV_PATH_ZEROCOPY),
+                          ("ce2d", B.KV_PATH_CE2D)):
+            pool.kv_pool_set_path(pid, pid)
+            ts = []
+            for k in range(45):
+                t0 = time.perf_counter()
+                pool.kv_rotate(og, oh, ih, ig)
+                pool.kv_sync()
+                if k >= 5:
+                    ts.append((time.perf_counter() - t0) * 1e6)
+            rec[name + "_us"] = round(float(np.median(ts)), 1)
+            if name == "auto":
+                rec["auto_took"] = B.PATH_NAMES[pool.kv_get_stats()["last_path_out"]]
+        rec["link_floor_us"] = round(n * shape.block_bytes / 50e9 * 1e6, 1)       # payload at 50 GB/s per direction
+        rows.append(rec)
+        _emit(rec, out)
+    pool.destroy()
+    print("\n| blocks each way | MiB each way | AUTO us (took) | staged us | zero-copy us | 2-D per block us | payload at 50 GB/s per direction, us |\n|---|---|---|---|---|---|---|")
+    for r in rows:
+        print(f"| {r['blocks_each_way']} | {r['mib_each_way']:g} | {r['auto_us']} ({r['auto_took']}) | {r['staged_us']} | {r['zerocopy_us']} | {r['ce2d_us']} | {r['link_floor_us']} |")
+
+
 def main() -> None:
     ap = argparse.ArgumentParser()
-    ap.add_argument("what", choices=["probe", "paths", "overlap"])
+    ap.add_argument("what", choices=["probe", "paths", "overlap", "latency"])
     ap.add_argument("--out", default=None)
     ap.add_argument("--max-payload-gb", type=float, default=4.0)
     ap.add_argument("--device-layout", choices=["layer-first", "block-first"], default="layer-first",
@@ -217,8 +258,10 @@ def main() -> None:
         probe(out)
     elif a.what == "paths":
         paths(out, a.max_payload_gb, 1 if a.device_layout == "block-first" else 0)
-    else:
+    elif a.what == "overlap":
         overlap(out)
+    else:
+        latency(out)
 
 
 if __name__ == "__main__":
