@@ -22,6 +22,12 @@
         host clock around kv_rotate + kv_sync, median of 40, per path.  What a per-request rotate costs
         when the link is not the limit.
 
+    python -m paper_2601_20309_b200.sweep budget [--b-xfer N] [--out FILE]
+        The serving replay (8B shape, 8 requests/s, 2000 steps) re-timed under the paper's per-iteration
+        transfer budget (B_xfer blocks per step, 2400 in the paper's main runs; remainder carried over):
+        device time of every step's rotation, against the 70 ms a model step takes in the paper
+        (section 5.3.4), i.e. how often the transfer would not hide behind the step.
+
 All print one JSON object per line and, at the end, a markdown table.
 """
 from __future__ import annotations
@@ -242,11 +248,46 @@ def latency(out) -> None:
         print(f"| {r['blocks_each_way']} | {r['mib_each_way']:g} | {r['auto_us']} ({r['auto_took']}) | {r['staged_us']} | {r['zerocopy_us']} | {r['ce2d_us']} | {r['link_floor_us']} |")
 
 
+def budget(out, b_xfer: int) -> None:
+    import numpy as np
+    import torch
+    w = W.config5_replay(rate=8.0)
+    shape = w.shape
+    steps = W.budgeted_steps(w.steps, b_xfer)
+    dev = torch.empty(w.nb_gpu * shape.block_bytes, dtype=torch.uint8, device="cuda:0")
+    pool = B.KVPool(shape.num_layers, shape.block_size, shape.kv_heads, shape.head_dim, w.nb_gpu, w.nb_host,
+                    dev.data_ptr())
+    ms, blocks = [], []
+    for r in steps:
+        if r.n_out + r.n_in == 0:
+            continue
+        pool.kv_rotate(r.out_gpu, r.out_host, r.in_host, r.in_gpu)
+        pool.kv_sync()
+        ms.append(pool.kv_get_stats()["last_union_ms"])
+        blocks.append(r.n_out + r.n_in)
+    pool.destroy()
+    ms, blocks = np.array(ms), np.array(blocks)
+    full = blocks >= b_xfer
+    rec = {"b_xfer": b_xfer, "original_steps": len(w.steps), "emitted_steps": len(steps), "steps_that_move_blocks": len(ms),
+           "blocks_moved": int(blocks.sum()), "steps_at_budget": int(full.sum()),
+           "ms_median": round(float(np.median(ms)), 2), "ms_p99": round(float(np.percentile(ms, 99)), 2),
+           "ms_max": round(float(ms.max()), 2), "ms_median_at_budget": round(float(np.median(ms[full])), 2) if full.any() else None,
+           "gbs_at_budget": round(float(np.median(blocks[full] * shape.block_bytes / ms[full] / 1e6)), 1) if full.any() else None,
+           "steps_over_70ms": int((ms > 70.0).sum()), "share_over_70ms": round(float((ms > 70.0).mean()), 4)}
+    _emit(rec, out)
+    print("\n| B_xfer | emitted steps | steps that move blocks | at budget | median ms | p99 ms | max ms | median ms at budget | "
+          "GB/s at budget | steps over 70 ms |\n|---|---|---|---|---|---|---|---|---|---|")
+    print(f"| {b_xfer} | {rec['emitted_steps']} | {rec['steps_that_move_blocks']} | {rec['steps_at_budget']} | {rec['ms_median']} | "
+          f"{rec['ms_p99']} | {rec['ms_max']} | {rec['ms_median_at_budget']} | {rec['gbs_at_budget']} | "
+          f"{rec['steps_over_70ms']} ({100 * rec['share_over_70ms']:.2f} %) |")
+
+
 def main() -> None:
     ap = argparse.ArgumentParser()
-    ap.add_argument("what", choices=["probe", "paths", "overlap", "latency"])
+    ap.add_argument("what", choices=["probe", "paths", "overlap", "latency", "budget"])
     ap.add_argument("--out", default=None)
     ap.add_argument("--max-payload-gb", type=float, default=4.0)
+    ap.add_argument("--b-xfer", type=int, default=2400, help="budget: blocks per step, both directions together")
     ap.add_argument("--device-layout", choices=["layer-first", "block-first"], default="layer-first",
                     help="paths: device pool layout (block-first = the paper's redesigned storage order)")
     a = ap.parse_args()
@@ -260,8 +301,10 @@ def main() -> None:
         paths(out, a.max_payload_gb, 1 if a.device_layout == "block-first" else 0)
     elif a.what == "overlap":
         overlap(out)
-    else:
+    elif a.what == "latency":
         latency(out)
+    else:
+        budget(out, a.b_xfer)
 
 
 if __name__ == "__main__":

@@ -546,3 +546,51 @@ def config5_replay(seed: int = MASTER_SEED + 5, rate: float = 16.0, n_steps: int
             remaining[rid] -= 1
     return Workload(f"replay_{rate:g}rps", shape, nb_gpu, nb_host, seed, tab, steps,
                     {"demand_blocks": demand, "arrivals": n_arr})
+
+
+# --------------------------------------------------------------------------- transfer budget per step
+
+def budgeted_steps(steps: Sequence[Rotation], b_xfer: int) -> List[Rotation]:
+    """Re-time a list of rotations under a per-step transfer budget of ``b_xfer`` blocks (both directions
+    together; the paper's scheduler bounds what one iteration may move by such a budget, 2400 blocks in
+    its main runs, so that the transfer hides behind one model step).  Work that does not fit a step is
+    carried over: the pairs of the incoming rotations are queued in arrival order (inside one rotation
+    swap-outs and swap-ins alternate, so both directions stay busy) and every emitted step takes pairs
+    from the front of the queue until the budget is used up, or until the next pair names a block that
+    a pair of the other direction already taken for this step names too, or a destination already
+    taken (a swap-in into device blocks that an earlier rotation's swap-out releases has to wait for the
+    next step: one rotate call must not overlap across directions, nor write a block twice).  The queue is never reordered, so the emitted steps do to the pools
+    exactly what the original ones did.  One emitted step per original step at least (idle steps stay),
+    more at the end until the queue is empty."""
+    assert b_xfer >= 1
+    queue: List[Tuple[int, int, int]] = []     # (direction 0 = out / 1 = in, gpu id, host id)
+    out: List[Rotation] = []
+
+    def emit():
+        taken = 0
+        g_used = (set(), set())                # device / host ids named so far, per direction
+        h_used = (set(), set())
+        while taken < len(queue) and taken < b_xfer:
+            d, g, h = queue[taken]
+            if g in g_used[1 - d] or h in h_used[1 - d] or (h in h_used[0] if d == 0 else g in g_used[1]):
+                break                          # other direction names it too, or a destination would repeat
+            g_used[d].add(g)
+            h_used[d].add(h)
+            taken += 1
+        part = queue[:taken]
+        del queue[:taken]
+        po = [p for p in part if p[0] == 0]
+        pi = [p for p in part if p[0] == 1]
+        z = np.zeros(1, np.int64)
+        out.append(Rotation(_i32([p[1] for p in po]), _i32([p[2] for p in po]), _i32([p[2] for p in pi]),
+                            _i32([p[1] for p in pi]), z, z.copy()))
+
+    for r in steps:
+        outs = [(0, int(g), int(h)) for g, h in zip(r.out_gpu, r.out_host)]
+        ins = [(1, int(g), int(h)) for h, g in zip(r.in_host, r.in_gpu)]
+        k = min(len(outs), len(ins))
+        queue += [p for pair in zip(outs[:k], ins[:k]) for p in pair] + outs[k:] + ins[k:]
+        emit()
+    while queue:
+        emit()
+    return out

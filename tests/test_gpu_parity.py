@@ -393,3 +393,18 @@ def test_stream_wait_orders_a_consumer_stream_behind_the_swap_in():
         p.assert_equal("after stream wait")
     finally:
         p.close()
+
+
+def test_budgeted_replay_matches_the_oracle():
+    """The replay lists re-timed under a per-step budget of 24 blocks (work carried over to later steps),
+    queued without syncing: same final pools as the oracle fed the same budgeted steps."""
+    w = W.config5_replay(rate=2.0, n_steps=300, shape=W.KVShape(2, 16, 2, 64), duration_s=20.0, max_tokens=1024)
+    steps = W.budgeted_steps(w.steps, 24)
+    assert len(steps) > len(w.steps) and max(s.n_out + s.n_in for s in steps) <= 24
+    p = _pair(w.shape, w.nb_gpu, w.nb_host, seed=w.seed)
+    try:
+        for r in steps:
+            assert p.rotate_both(r) == 0
+        p.assert_equal("budgeted replay")
+    finally:
+        p.close()

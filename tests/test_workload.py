@@ -99,3 +99,26 @@ def test_config5_replay_interleaves_and_stays_consistent():
         assert not set(s.in_gpu) & set(s.out_gpu) and not set(s.in_host) & set(s.out_host)
         assert len(set(s.in_gpu)) == s.n_in and len(set(s.out_host)) == s.n_out
     w.table.check_consistent()
+
+
+def test_budgeted_steps_respect_the_budget_and_change_nothing_else():
+    """Re-timing rotations under a per-step block budget: no step moves more than the budget, nothing is
+    lost or reordered inside a direction, and the pools end up as with the original steps."""
+    from oracle.kv_definition import TagModel
+    w = W.config5_replay(rate=2.0, n_steps=300, shape=W.KVShape(2, 16, 2, 64), duration_s=20.0, max_tokens=1024)
+    for b_xfer in (7, 24, 10_000):
+        steps = W.budgeted_steps(w.steps, b_xfer)
+        assert len(steps) >= len(w.steps)
+        assert max(s.n_out + s.n_in for s in steps) <= b_xfer
+        cat = lambda xs: np.concatenate(xs) if xs else np.empty(0, np.int32)
+        for field in ("out_gpu", "out_host", "in_host", "in_gpu"):
+            assert np.array_equal(cat([getattr(s, field) for s in steps]), cat([getattr(s, field) for s in w.steps]))
+        a, b = TagModel(w.nb_gpu, w.nb_host), TagModel(w.nb_gpu, w.nb_host)
+        for s in w.steps:
+            assert a.rotate(s.out_gpu.tolist(), s.out_host.tolist(), s.in_host.tolist(), s.in_gpu.tolist()) == 0
+        for s in steps:     # every emitted step is itself a valid rotation (no cross-direction overlap)
+            assert b.rotate(s.out_gpu.tolist(), s.out_host.tolist(), s.in_host.tolist(), s.in_gpu.tolist()) == 0
+        assert a.g_tag == b.g_tag and a.h_tag == b.h_tag
+    if True:
+        big = W.budgeted_steps(w.steps, 10_000)
+        assert len(big) == len(w.steps) and all(x.n_out == y.n_out and x.n_in == y.n_in for x, y in zip(big, w.steps))
