@@ -21,6 +21,7 @@ namespace {
 constexpr int KV_SLOTS = 8;            // descriptor / event ring depth per direction
 constexpr int KV_MAX_CE_STREAMS = 4;
 constexpr int64_t KV_AUTO_MIN_TRANSFER = 3ll << 20;   // AUTO: staged when its transfers average 3 MiB or more
+constexpr int64_t KV_MERGE_MIN_MEAN_RUN = 8;          // STAGED: merge runs of host ids when they average 8 blocks or more
 constexpr int BULK_STAGE = 16384;      // bytes per shared-memory stage of the bulk kernel
 constexpr int BULK_NS = 8;             // stages
 constexpr int BULK_AHEAD = 5;          // loads in flight ahead of the stores
@@ -40,6 +41,8 @@ thread_local char g_err[256] = "";
 struct CeOp {
     int64_t host_off, stage_off, width, host_pitch;
     int32_t rows;
+    int64_t pos;        // planning: where its blocks start in the list sorted by host id
+    int32_t nblk;       // blocks it moves (rows x blocks per row)
 };
 // Sorted list positions [lo, hi) go through one staging half; ops [op_lo, op_hi) move them.
 struct CeChunk {
@@ -68,7 +71,7 @@ struct DirState {
     std::vector<cudaEvent_t> kev;
     std::vector<int64_t> kev_bytes;
     int kev_used = 0;
-    std::vector<int32_t> order;        // list positions sorted by host id
+    std::vector<int32_t> order;        // list positions sorted by host id (= staging order)
     std::vector<CeOp> ops;             // transfers of the current call, in issue order
     std::vector<CeChunk> chunks;       // the call cut into staging-half-sized pieces
     int ctas = 0;
@@ -335,9 +338,9 @@ int32_t ce_join(kv_pool *p, DirState &s)
     return KV_OK;
 }
 
-// STAGED path, host side of one direction of one call: sort the pairs by host id so that blocks that
-// are neighbours in host memory become one transfer, cut the sorted list into staging-half-sized
-// chunks, and turn every chunk into as few copy-engine transfers as its host ids allow.
+// STAGED path, host side of one direction of one call: sort the pairs by host id, turn the sorted list
+// into copy-engine transfers (long ones where the host ids form long runs, uniform two-block ones
+// otherwise), and cut that sequence into chunks of at most a staging half.
 //   - a run of consecutive host ids is one plain transfer;
 //   - runs of equal length whose starts are equally spaced become one strided 2-D transfer (any two
 //     runs are "equally spaced", so isolated blocks still travel two per transfer).
@@ -354,46 +357,77 @@ int32_t plan_staged(kv_pool *p, DirCall &c)
             std::sort(s.order.begin(), s.order.end(), [&](int32_t a, int32_t b) { return c.host_ids[a] < c.host_ids[b]; });
         s.ops.clear();
         s.chunks.clear();
-        // The first chunk of a swap-out is half as long as the rest: its first transfer starts sooner, and
-        // in a rotation the pack kernels then run midway between the swap-in's unpack kernels instead of
-        // at the same moments (both directions advance one chunk per equal stretch of link time).
         // A call that would fit one half is still cut into about four chunks (of 8 MiB or more), so that its
-        // own packing, transfers and unpacking overlap instead of following one another.
+        // own packing, transfers and unpacking overlap instead of following one another.  The first chunk
+        // of a swap-out is half as long as the rest: its first transfer starts sooner.
         const int64_t min_chunk = std::max<int64_t>(1, (8ll << 20) / p->blk);
         const int64_t chunk = std::min(s.half_blocks, std::max(min_chunk, (c.n + 3) / 4));
         const int64_t first = (c.d == 0 && c.n > chunk) ? std::max<int64_t>(1, chunk / 2) : chunk;
-        for (int64_t lo = 0, hi = 0; lo < c.n; lo = hi) {
-            hi = std::min(c.n, lo + (lo == 0 ? first : chunk));
-            CeChunk ch{lo, hi, (int32_t)s.ops.size(), 0};
-            if (layer_first) {
-                // one strided transfer per block: `planes` rows of SEG bytes, a whole host plane apart
+        if (layer_first) {
+            // one strided transfer per block: `planes` rows of SEG bytes, a whole host plane apart
+            for (int64_t lo = 0, hi = 0; lo < c.n; lo = hi) {
+                hi = std::min(c.n, lo + (lo == 0 ? first : chunk));
+                CeChunk ch{lo, hi, (int32_t)s.ops.size(), 0};
                 for (int64_t k = lo; k < hi; ++k)
                     s.ops.push_back(CeOp{(int64_t)c.host_ids[s.order[(size_t)k]] * p->seg, (k - lo) * p->blk, p->seg,
-                                         p->cfg.num_host_blocks * p->seg, p->planes});
-            } else {
-                int64_t k = lo;
-                auto hid = [&](int64_t q) { return (int64_t)c.host_ids[s.order[(size_t)q]]; };
-                auto run_len = [&](int64_t q) {
-                    int64_t r = 1;
-                    while (q + r < hi && hid(q + r) == hid(q) + r) ++r;
-                    return r;
-                };
-                while (k < hi) {
-                    const int64_t r = run_len(k);
-                    CeOp op{hid(k) * p->blk, (k - lo) * p->blk, r * p->blk, r * p->blk, 1};
-                    int64_t nxt = k + r;
-                    // further runs of the same length at a constant spacing join as extra rows
-                    while (nxt < hi && run_len(nxt) == r) {
-                        const int64_t pitch = (hid(nxt) - hid(nxt - r)) * p->blk;
-                        if (pitch < op.width || pitch > p->max_pitch || (op.rows > 1 && pitch != op.host_pitch)) break;
-                        op.host_pitch = pitch;
-                        op.rows++;
-                        nxt += r;
-                    }
-                    s.ops.push_back(op);
-                    k = nxt;
-                }
+                                         p->cfg.num_host_blocks * p->seg, p->planes, k, 1});
+                ch.op_hi = (int32_t)s.ops.size();
+                s.chunks.push_back(ch);
             }
+            c.planned = true;
+            return KV_OK;
+        }
+        // ---- 1. transfers over the sorted list, none longer than a chunk.
+        // Measured with both directions busy: transfers that all carry the same number of bytes keep the
+        // two copy engines in step and share the link evenly (2 x 2 MiB everywhere: 93.9 GB/s), while a
+        // mix of sizes loses 8 % (85.6 GB/s for mostly pairs with a few singles and triples), whatever
+        // the order of issue.  Merging neighbouring host blocks into long transfers only pays once the
+        // runs are long (mean of 8 blocks and more: 89 to 99 GB/s); below that every block is treated
+        // as a single and sent with its neighbour in the sorted list, two per transfer, all alike.
+        auto hid = [&](int64_t q) { return (int64_t)c.host_ids[s.order[(size_t)q]]; };
+        int64_t nruns = 1;
+        for (int64_t q = 1; q < c.n; ++q)
+            if (hid(q) != hid(q - 1) + 1) ++nruns;
+        const bool uniform = c.n < KV_MERGE_MIN_MEAN_RUN * nruns;
+        auto run_len = [&](int64_t q) {
+            int64_t r = 1;
+            if (uniform) return r;
+            while (q + r < c.n && r < chunk && hid(q + r) == hid(q) + r) ++r;
+            return r;
+        };
+        for (int64_t k = 0; k < c.n;) {
+            const int64_t r = run_len(k);
+            CeOp op{hid(k) * p->blk, 0, r * p->blk, r * p->blk, 1, k, (int32_t)r};
+            int64_t nxt = k + r;
+            // further runs of the same length at a constant spacing join as extra rows (uniform mode: one)
+            while (nxt < c.n && op.nblk + r <= chunk && run_len(nxt) == r && !(uniform && op.rows >= 2)) {
+                const int64_t pitch = (hid(nxt) - hid(nxt - r)) * p->blk;
+                if (pitch < op.width || pitch > p->max_pitch || (op.rows > 1 && pitch != op.host_pitch)) break;
+                op.host_pitch = pitch;
+                op.rows++;
+                op.nblk += (int32_t)r;
+                nxt += r;
+            }
+            s.ops.push_back(op);
+            k = nxt;
+        }
+        // ---- 2. staging slots follow the sorted order; chunks are cut when a staging half is full
+        int64_t filled = 0;
+        CeChunk ch{0, 0, 0, 0};
+        for (size_t a = 0; a < s.ops.size(); ++a) {
+            CeOp &op = s.ops[a];
+            const int64_t cap = s.chunks.empty() ? first : chunk;
+            if (filled > ch.lo && filled - ch.lo + op.nblk > cap) {
+                ch.hi = filled;
+                ch.op_hi = (int32_t)a;
+                s.chunks.push_back(ch);
+                ch = CeChunk{filled, filled, (int32_t)a, 0};
+            }
+            op.stage_off = (filled - ch.lo) * p->blk;
+            filled += op.nblk;
+        }
+        if (filled > ch.lo) {
+            ch.hi = filled;
             ch.op_hi = (int32_t)s.ops.size();
             s.chunks.push_back(ch);
         }
