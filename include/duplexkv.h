@@ -170,6 +170,30 @@ int32_t kv_rotate(kv_pool_t *pool,
                   const int32_t *out_gpu, const int32_t *out_host, int64_t n_out,
                   const int32_t *in_host, const int32_t *in_gpu, int64_t n_in);
 
+/*
+ * What copy-engine transfers the STAGED path would make for one direction of a call (no pool, no GPU):
+ * the list is sorted by host id; where the ids form long runs (8 blocks and more on average) each run
+ * is one transfer and equal runs at a constant spacing share one strided transfer; otherwise every
+ * transfer carries exactly two blocks (neighbours in the sorted list, any distance apart in host
+ * memory), because transfers of one size keep the two copy engines of a rotation in step (section
+ * 4.3.2's "merge small segments into large transfers", bounded here by what the ids allow).  The sequence
+ * is cut into chunks of at most half_blocks blocks (one staging half each; about four chunks for a
+ * call that would fit one half).
+ *   host_ids   HOST array of n host block ids (direction 0: swap-out destinations, 1: swap-in sources)
+ *   ops        HOST array of ops_cap entries, filled in issue order; *n_ops = transfers needed
+ *              (with ops_cap == 0 only the count is returned)
+ *   order      HOST array of n entries or NULL: order[k] = index in host_ids of the block that takes
+ *              staging position k (= position k of the sorted list)
+ * A transfer moves rows x blocks_per_row blocks: row r covers host blocks host_block + r*pitch_blocks ..
+ * + blocks_per_row - 1 and staging positions first_position + r*blocks_per_row .. of the sorted list.
+ */
+typedef struct {
+    int64_t host_block, first_position, pitch_blocks;
+    int32_t rows, blocks_per_row, chunk, pad_;
+} kv_plan_op_t;
+int32_t kv_plan_staged(int64_t blk_bytes, int64_t half_blocks, int32_t direction, const int32_t *host_ids, int64_t n,
+                       kv_plan_op_t *ops, int64_t ops_cap, int64_t *n_ops, int32_t *order);
+
 /* Wait for outstanding work, then change the transfer path of each direction (KV_PATH_*; AUTO
  * re-applies the rule of kv_path_for).  Pool contents are unaffected. */
 int32_t kv_pool_set_path(kv_pool_t *pool, int32_t path_out, int32_t path_in);

@@ -92,10 +92,15 @@ class kv_table_stats_t(C.Structure):
                                          "requests")]
 
 
+class kv_plan_op_t(C.Structure):
+    _fields_ = [("host_block", C.c_int64), ("first_position", C.c_int64), ("pitch_blocks", C.c_int64),
+                ("rows", C.c_int32), ("blocks_per_row", C.c_int32), ("chunk", C.c_int32), ("pad_", C.c_int32)]
+
+
 EXPORTS = ["kv_pool_create", "kv_pool_destroy", "kv_pool_set_path", "kv_swap_out", "kv_swap_in", "kv_rotate", "kv_sync",
            "kv_gather_blocks", "kv_scatter_blocks", "kv_host_ptr", "kv_get_stats", "kv_last_error",
            "kv_seg_bytes", "kv_blk_bytes", "kv_path_for", "kv_probe_link", "kv_probe_link_ex",
-           "kv_gather_blocks_static", "kv_pool_shape", "kv_pool_progress", "kv_stream_wait",
+           "kv_gather_blocks_static", "kv_pool_shape", "kv_pool_progress", "kv_stream_wait", "kv_plan_staged",
            "kv_table_create", "kv_table_create_dry", "kv_table_destroy", "kv_table_last_error", "kv_req_add",
            "kv_req_append", "kv_eager_rotate", "kv_req_rotate", "kv_req_preempt", "kv_req_resume", "kv_req_finish",
            "kv_req_info", "kv_req_blocks", "kv_table_get_stats"]
@@ -146,6 +151,8 @@ def lib() -> C.CDLL:
     i64p = C.POINTER(C.c_int64)
     L.kv_pool_shape.restype = C.c_int32
     L.kv_pool_shape.argtypes = [vp, C.POINTER(kv_pool_shape_t)]
+    L.kv_plan_staged.restype = C.c_int32
+    L.kv_plan_staged.argtypes = [i64, i64, C.c_int32, i32p, i64, C.POINTER(kv_plan_op_t), i64, i64p, i32p]
     L.kv_stream_wait.restype = C.c_int32
     L.kv_stream_wait.argtypes = [vp, vp, C.c_int32]
     L.kv_pool_progress.restype = C.c_int32
@@ -227,6 +234,21 @@ def kv_probe_link_ex(device_id: int, copy_bytes: int, total_bytes: int, span_byt
     if rc != KV_OK:
         raise KVError(rc, lib().kv_last_error(None).decode())
     return {k: getattr(out, k) for k, _ in kv_link_probe_t._fields_ if k != "pad_"}
+
+
+def kv_plan_staged(blk_bytes: int, half_blocks: int, direction: int, host_ids):
+    """(ops, order): the transfers the STAGED path would make for these host ids, as a list of dicts in
+    issue order, and the staging order as a numpy array of indices into ``host_ids``.  Needs no GPU."""
+    h, hp = _ids(host_ids)
+    n_ops = C.c_int64()
+    ops = (kv_plan_op_t * max(1, len(h)))()
+    order = np.empty(len(h), np.int32)
+    rc = lib().kv_plan_staged(blk_bytes, half_blocks, direction, hp, len(h), ops, len(ops), C.byref(n_ops),
+                              order.ctypes.data_as(C.POINTER(C.c_int32)))
+    if rc != KV_OK:
+        raise KVError(rc, lib().kv_last_error(None).decode())
+    fields = [k for k, _ in kv_plan_op_t._fields_ if k != "pad_"]
+    return [{k: getattr(ops[a], k) for k in fields} for a in range(n_ops.value)], order
 
 
 KV_STATIC_MAX_BLOCKS = 8192

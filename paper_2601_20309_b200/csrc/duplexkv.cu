@@ -346,36 +346,42 @@ int32_t ce_join(kv_pool *p, DirState &s)
 //     runs are "equally spaced", so isolated blocks still travel two per transfer).
 // The cost of a transfer on the copy engine is a fixed start-up plus its bytes, so fewer and larger
 // transfers are what keeps the link busy.
-int32_t plan_staged(kv_pool *p, DirCall &c)
+struct PlanParams {
+    int64_t blk, seg, half_blocks, max_pitch, num_host_blocks;
+    int planes;
+    bool layer_first;           // host pool layout
+};
+
+// Pure planning (no pool, no CUDA): order, transfers and chunks for n pairs of direction d (0 out, 1 in)
+// whose host block ids are host_ids.  May throw std::bad_alloc.
+void plan_transfers(const PlanParams &pp, int d, const int32_t *host_ids, int64_t n, std::vector<int32_t> &order,
+                    std::vector<CeOp> &ops, std::vector<CeChunk> &chunks)
 {
-    DirState &s = p->dir[c.d];
-    const bool layer_first = p->cfg.host_layout == KV_HOST_LAYER_FIRST;
-    try {
-        s.order.resize((size_t)c.n);
-        for (int64_t i = 0; i < c.n; ++i) s.order[(size_t)i] = (int32_t)i;
-        if (!layer_first)
-            std::sort(s.order.begin(), s.order.end(), [&](int32_t a, int32_t b) { return c.host_ids[a] < c.host_ids[b]; });
-        s.ops.clear();
-        s.chunks.clear();
+    {
+        order.resize((size_t)n);
+        for (int64_t i = 0; i < n; ++i) order[(size_t)i] = (int32_t)i;
+        if (!pp.layer_first)
+            std::sort(order.begin(), order.end(), [&](int32_t a, int32_t b) { return host_ids[a] < host_ids[b]; });
+        ops.clear();
+        chunks.clear();
         // A call that would fit one half is still cut into about four chunks (of 8 MiB or more), so that its
         // own packing, transfers and unpacking overlap instead of following one another.  The first chunk
         // of a swap-out is half as long as the rest: its first transfer starts sooner.
-        const int64_t min_chunk = std::max<int64_t>(1, (8ll << 20) / p->blk);
-        const int64_t chunk = std::min(s.half_blocks, std::max(min_chunk, (c.n + 3) / 4));
-        const int64_t first = (c.d == 0 && c.n > chunk) ? std::max<int64_t>(1, chunk / 2) : chunk;
-        if (layer_first) {
+        const int64_t min_chunk = std::max<int64_t>(1, (8ll << 20) / pp.blk);
+        const int64_t chunk = std::min(pp.half_blocks, std::max(min_chunk, (n + 3) / 4));
+        const int64_t first = (d == 0 && n > chunk) ? std::max<int64_t>(1, chunk / 2) : chunk;
+        if (pp.layer_first) {
             // one strided transfer per block: `planes` rows of SEG bytes, a whole host plane apart
-            for (int64_t lo = 0, hi = 0; lo < c.n; lo = hi) {
-                hi = std::min(c.n, lo + (lo == 0 ? first : chunk));
-                CeChunk ch{lo, hi, (int32_t)s.ops.size(), 0};
+            for (int64_t lo = 0, hi = 0; lo < n; lo = hi) {
+                hi = std::min(n, lo + (lo == 0 ? first : chunk));
+                CeChunk ch{lo, hi, (int32_t)ops.size(), 0};
                 for (int64_t k = lo; k < hi; ++k)
-                    s.ops.push_back(CeOp{(int64_t)c.host_ids[s.order[(size_t)k]] * p->seg, (k - lo) * p->blk, p->seg,
-                                         p->cfg.num_host_blocks * p->seg, p->planes, k, 1});
-                ch.op_hi = (int32_t)s.ops.size();
-                s.chunks.push_back(ch);
+                    ops.push_back(CeOp{(int64_t)host_ids[order[(size_t)k]] * pp.seg, (k - lo) * pp.blk, pp.seg,
+                                         pp.num_host_blocks * pp.seg, pp.planes, k, 1});
+                ch.op_hi = (int32_t)ops.size();
+                chunks.push_back(ch);
             }
-            c.planned = true;
-            return KV_OK;
+            return;
         }
         // ---- 1. transfers over the sorted list, none longer than a chunk.
         // Measured with both directions busy: transfers that all carry the same number of bytes keep the
@@ -384,53 +390,63 @@ int32_t plan_staged(kv_pool *p, DirCall &c)
         // the order of issue.  Merging neighbouring host blocks into long transfers only pays once the
         // runs are long (mean of 8 blocks and more: 89 to 99 GB/s); below that every block is treated
         // as a single and sent with its neighbour in the sorted list, two per transfer, all alike.
-        auto hid = [&](int64_t q) { return (int64_t)c.host_ids[s.order[(size_t)q]]; };
+        auto hid = [&](int64_t q) { return (int64_t)host_ids[order[(size_t)q]]; };
         int64_t nruns = 1;
-        for (int64_t q = 1; q < c.n; ++q)
+        for (int64_t q = 1; q < n; ++q)
             if (hid(q) != hid(q - 1) + 1) ++nruns;
-        const bool uniform = c.n < KV_MERGE_MIN_MEAN_RUN * nruns;
+        const bool uniform = n < KV_MERGE_MIN_MEAN_RUN * nruns;
         auto run_len = [&](int64_t q) {
             int64_t r = 1;
             if (uniform) return r;
-            while (q + r < c.n && r < chunk && hid(q + r) == hid(q) + r) ++r;
+            while (q + r < n && r < chunk && hid(q + r) == hid(q) + r) ++r;
             return r;
         };
-        for (int64_t k = 0; k < c.n;) {
+        for (int64_t k = 0; k < n;) {
             const int64_t r = run_len(k);
-            CeOp op{hid(k) * p->blk, 0, r * p->blk, r * p->blk, 1, k, (int32_t)r};
+            CeOp op{hid(k) * pp.blk, 0, r * pp.blk, r * pp.blk, 1, k, (int32_t)r};
             int64_t nxt = k + r;
             // further runs of the same length at a constant spacing join as extra rows (uniform mode: one)
-            while (nxt < c.n && op.nblk + r <= chunk && run_len(nxt) == r && !(uniform && op.rows >= 2)) {
-                const int64_t pitch = (hid(nxt) - hid(nxt - r)) * p->blk;
-                if (pitch < op.width || pitch > p->max_pitch || (op.rows > 1 && pitch != op.host_pitch)) break;
+            while (nxt < n && op.nblk + r <= chunk && run_len(nxt) == r && !(uniform && op.rows >= 2)) {
+                const int64_t pitch = (hid(nxt) - hid(nxt - r)) * pp.blk;
+                if (pitch < op.width || pitch > pp.max_pitch || (op.rows > 1 && pitch != op.host_pitch)) break;
                 op.host_pitch = pitch;
                 op.rows++;
                 op.nblk += (int32_t)r;
                 nxt += r;
             }
-            s.ops.push_back(op);
+            ops.push_back(op);
             k = nxt;
         }
         // ---- 2. staging slots follow the sorted order; chunks are cut when a staging half is full
         int64_t filled = 0;
         CeChunk ch{0, 0, 0, 0};
-        for (size_t a = 0; a < s.ops.size(); ++a) {
-            CeOp &op = s.ops[a];
-            const int64_t cap = s.chunks.empty() ? first : chunk;
+        for (size_t a = 0; a < ops.size(); ++a) {
+            CeOp &op = ops[a];
+            const int64_t cap = chunks.empty() ? first : chunk;
             if (filled > ch.lo && filled - ch.lo + op.nblk > cap) {
                 ch.hi = filled;
                 ch.op_hi = (int32_t)a;
-                s.chunks.push_back(ch);
+                chunks.push_back(ch);
                 ch = CeChunk{filled, filled, (int32_t)a, 0};
             }
-            op.stage_off = (filled - ch.lo) * p->blk;
+            op.stage_off = (filled - ch.lo) * pp.blk;
             filled += op.nblk;
         }
         if (filled > ch.lo) {
             ch.hi = filled;
-            ch.op_hi = (int32_t)s.ops.size();
-            s.chunks.push_back(ch);
+            ch.op_hi = (int32_t)ops.size();
+            chunks.push_back(ch);
         }
+    }
+}
+
+int32_t plan_staged(kv_pool *p, DirCall &c)
+{
+    DirState &s = p->dir[c.d];
+    const PlanParams pp{p->blk, p->seg, s.half_blocks, p->max_pitch, p->cfg.num_host_blocks, p->planes,
+                        p->cfg.host_layout == KV_HOST_LAYER_FIRST};
+    try {
+        plan_transfers(pp, c.d, c.host_ids, c.n, s.order, s.ops, s.chunks);
     } catch (...) {
         return fail(p, KV_ERR_NOMEM, "out of host memory");
     }
@@ -1067,6 +1083,43 @@ int32_t kv_rotate(kv_pool_t *p, const int32_t *out_gpu, const int32_t *out_host,
     rc = run_calls(p, &late, 1, &wait_late, false);
     p->union_slot[0] = out_slot;
     return rc;
+}
+
+int32_t kv_plan_staged(int64_t blk_bytes, int64_t half_blocks, int32_t direction, const int32_t *host_ids, int64_t n,
+                       kv_plan_op_t *ops, int64_t ops_cap, int64_t *n_ops, int32_t *order)
+{
+    if (n_ops) *n_ops = 0;
+    if (blk_bytes <= 0 || half_blocks <= 0 || (direction != 0 && direction != 1) || n < 0 || (n && !host_ids) || !n_ops ||
+        (ops_cap && !ops))
+        return fail(nullptr, KV_ERR_INVALID_ARG, "bad planning arguments");
+    for (int64_t i = 0; i < n; ++i)
+        if (host_ids[i] < 0) return fail(nullptr, KV_ERR_RANGE, "negative host id");
+    std::vector<int32_t> ord;
+    std::vector<CeOp> v;
+    std::vector<CeChunk> ch;
+    const PlanParams pp{blk_bytes, blk_bytes, half_blocks, (int64_t)INT32_MAX, 0, 1, false};
+    try {
+        if (n) plan_transfers(pp, direction, host_ids, n, ord, v, ch);
+    } catch (...) {
+        return fail(nullptr, KV_ERR_NOMEM, "out of host memory");
+    }
+    *n_ops = (int64_t)v.size();
+    if ((int64_t)v.size() > ops_cap) return ops_cap ? fail(nullptr, KV_ERR_INVALID_ARG, "ops array too short") : KV_OK;
+    for (size_t q = 0; q < ch.size(); ++q)
+        for (int32_t a = ch[q].op_lo; a < ch[q].op_hi; ++a) {
+            const CeOp &o = v[(size_t)a];
+            kv_plan_op_t &r = ops[a];
+            r.host_block = o.host_off / blk_bytes;
+            r.first_position = o.pos;
+            r.rows = o.rows;
+            r.blocks_per_row = (int32_t)(o.width / blk_bytes);
+            r.pitch_blocks = o.rows > 1 ? o.host_pitch / blk_bytes : r.blocks_per_row;
+            r.chunk = (int32_t)q;
+            r.pad_ = 0;
+        }
+    if (order)
+        for (int64_t i = 0; i < n; ++i) order[i] = ord[(size_t)i];
+    return KV_OK;
 }
 
 int32_t kv_pool_set_path(kv_pool_t *p, int32_t path_out, int32_t path_in)

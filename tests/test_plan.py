@@ -1,0 +1,103 @@
+"""The staged path's transfer planner (host logic, no GPU): for any list of host ids the planned
+transfers cover every block exactly once, their row geometry matches the ids, no chunk exceeds a staging
+half, scattered lists give transfers that all carry two blocks, and long runs are merged."""
+import numpy as np
+import pytest
+
+from paper_2601_20309_b200 import binding as B
+
+BLK = 2 << 20
+
+
+def check_plan(host_ids, half_blocks, direction, blk=BLK):
+    host_ids = np.asarray(host_ids, np.int32)
+    ops, order = B.kv_plan_staged(blk, half_blocks, direction, host_ids)
+    n = len(host_ids)
+    assert sorted(order.tolist()) == list(range(n))                         # a permutation of the list
+    sorted_ids = host_ids[order]
+    assert np.all(np.diff(sorted_ids) >= 0)                                 # staging order = ascending host id
+    pos = 0
+    per_chunk = {}
+    for op in ops:
+        assert op["first_position"] == pos                                  # issue order walks the sorted list
+        assert op["rows"] >= 1 and op["blocks_per_row"] >= 1
+        for r in range(op["rows"]):
+            for j in range(op["blocks_per_row"]):
+                want = op["host_block"] + r * op["pitch_blocks"] + j
+                assert sorted_ids[pos] == want, (op, r, j)
+                pos += 1
+        if op["rows"] > 1:
+            assert op["pitch_blocks"] >= op["blocks_per_row"]                # rows do not overlap in host memory
+            assert op["pitch_blocks"] * blk <= 2 ** 31 - 1                   # what a strided transfer accepts
+        per_chunk[op["chunk"]] = per_chunk.get(op["chunk"], 0) + op["rows"] * op["blocks_per_row"]
+    assert pos == n                                                          # every block exactly once
+    assert sorted(per_chunk) == list(range(len(per_chunk)))                  # chunks numbered in order
+    assert all(v <= half_blocks for v in per_chunk.values())                 # a chunk fits a staging half
+    return ops, per_chunk
+
+
+@pytest.mark.parametrize("direction", [0, 1])
+@pytest.mark.parametrize("seed", range(5))
+def test_scattered_ids_travel_two_per_transfer_all_alike(seed, direction):
+    rng = np.random.default_rng(seed)
+    n = int(rng.integers(50, 700))
+    ids = rng.choice(60_000, n, replace=False)
+    ops, chunks = check_plan(ids, 512, direction)
+    sizes = [op["rows"] * op["blocks_per_row"] for op in ops]
+    # ids more than 2 GiB apart cannot share a strided transfer; everything else is a pair
+    assert sizes.count(2) >= len(sizes) - 1 - sum(1 for a, b in zip(np.sort(ids), np.sort(ids)[1:]) if (b - a) * BLK > 2 ** 31 - 1)
+    assert max(sizes) == 2
+    assert len(ops) <= (n + 1) // 2 + 8
+
+
+def test_long_runs_are_merged_and_cut_at_chunk_size():
+    ids = np.concatenate([np.arange(1000, 1300), np.arange(5000, 5200), np.arange(9000, 9040)])    # runs of 300, 200, 40
+    rng = np.random.default_rng(0)
+    ops, chunks = check_plan(rng.permutation(ids), 128, 1)
+    assert all(op["rows"] * op["blocks_per_row"] <= 128 for op in ops)
+    assert len(ops) <= 8                                                     # 300 -> 3, 200 -> 2, 40 -> 1 (or merged rows)
+    assert sum(chunks.values()) == 540
+    one, _ = check_plan(np.arange(77, 77 + 64), 512, 0)                      # a call that fits one half: about four chunks
+    assert 3 <= len({op["chunk"] for op in one}) <= 6
+
+
+def test_short_runs_are_not_merged_into_uneven_transfers():
+    """Runs of 1 to 4 blocks: merging would give transfers of many sizes; the plan keeps them all alike."""
+    rng = np.random.default_rng(3)
+    ids, at = [], 0
+    while len(ids) < 400:
+        L = int(rng.integers(1, 5))
+        ids += list(range(at, at + L))
+        at += L + int(rng.integers(2, 50))
+    ops, _ = check_plan(rng.permutation(np.array(ids[:400])), 512, 0)
+    assert {op["rows"] * op["blocks_per_row"] for op in ops} == {2}
+    assert len(ops) == 200
+
+
+def test_equal_runs_at_a_constant_spacing_share_one_strided_transfer():
+    ids = np.concatenate([np.arange(s, s + 16) for s in range(100, 100 + 8 * 40, 40)])            # 8 runs of 16, 40 apart
+    ops, _ = check_plan(ids, 512, 0)
+    assert any(op["rows"] > 1 and op["blocks_per_row"] == 16 and op["pitch_blocks"] == 40 for op in ops)
+    assert len(ops) <= 4
+
+
+def test_repeated_sources_far_apart_ids_and_tiny_lists():
+    check_plan([7, 7, 8, 7, 30, 30, 31], 16, 1)                              # swap-in sources may repeat
+    ops, _ = check_plan([0, 5000, 10000, 15000], 16, 0)                      # more than 2 GiB apart: singles
+    assert all(op["rows"] == 1 for op in ops)
+    ops, _ = check_plan([42], 16, 0)
+    assert len(ops) == 1
+    ops, order = B.kv_plan_staged(BLK, 16, 0, [])
+    assert ops == [] and len(order) == 0
+    check_plan(np.arange(50)[::-1], 3, 1)                                    # tiny staging halves
+    with pytest.raises(B.KVError):
+        B.kv_plan_staged(BLK, 0, 0, [1, 2])
+    with pytest.raises(B.KVError):
+        B.kv_plan_staged(BLK, 16, 0, [1, -2])
+
+
+@pytest.mark.parametrize("blk", [128 << 10, 1 << 20, 8 << 20])
+def test_other_block_sizes(blk):
+    rng = np.random.default_rng(9)
+    check_plan(rng.choice(5000, 333, replace=False), max(2, (64 << 20) // blk), 0, blk=blk)
+    check_plan(np.arange(10, 410), max(2, (64 << 20) // blk), 1, blk=blk)
