@@ -123,6 +123,8 @@ typedef struct {
     double  timed_kernel_ms;           /* KV_FLAG_TIME_KERNELS: summed device time of the timed kernels   */
     int64_t timed_kernel_bytes;        /* payload bytes those kernels moved (each read once, written once)*/
     int64_t timed_kernels;             /* how many launches the two sums cover                            */
+    double  timed_kernel_exec_ms;      /* the same launches timed from inside: earliest CTA start to latest
+                                          CTA end (%globaltimer), i.e. without the wait for the launch     */
 } kv_stats_t;
 
 typedef struct {

@@ -71,6 +71,7 @@ struct DirState {
     std::vector<cudaEvent_t> kev;
     std::vector<int64_t> kev_bytes;
     int kev_used = 0;
+    unsigned long long *ktime_dev = nullptr;   // 2 words per timed launch: earliest CTA start, latest CTA end
     std::vector<int32_t> order;        // list positions sorted by host id (= staging order)
     std::vector<CeOp> ops;             // transfers of the current call, in issue order
     std::vector<CeChunk> chunks;       // the call cut into staging-half-sized pieces
@@ -174,6 +175,7 @@ void fill_geometry(const kv_pool *p, KvJob &job, bool link = false)
     job.chunk = (int)std::min<int64_t>(p->seg, max_chunk);
     job.cps = (int)((p->seg + job.chunk - 1) / job.chunk);
     job.status = p->status_dev;
+    job.t_first = job.t_last = nullptr;
 }
 
 int clamp_ctas(const KvJob &job, const KvDir &d, int want)
@@ -199,11 +201,30 @@ cudaError_t launch_job(kv_pool *p, const KvJob &job, cudaStream_t stream, bool l
 
 constexpr int KV_MAX_TIMED = 2048;     // kernel launches per direction timed between two kv_sync calls
 
-// HBM-to-HBM gather / scatter launch, bracketed by events on its stream when kernel timing is on
-cudaError_t launch_timed(kv_pool *p, DirState &s, cudaStream_t stream, const KvJob &job, int64_t payload_bytes)
+// earliest-start words to all ones, latest-end words to zero (a strided 2-D memset each)
+cudaError_t preset_ktime(DirState &s, cudaStream_t stream)
+{
+    cudaError_t rc = cudaMemset2DAsync(s.ktime_dev, 16, 0xFF, 8, KV_MAX_TIMED, stream);
+    if (rc != cudaSuccess) return rc;
+    return cudaMemset2DAsync(s.ktime_dev + 1, 16, 0x00, 8, KV_MAX_TIMED, stream);
+}
+
+// HBM-to-HBM gather / scatter launch, bracketed by events on its stream when kernel timing is on, and
+// then also timed from inside (first CTA start to last CTA end), which leaves out the wait for the launch
+cudaError_t launch_timed(kv_pool *p, DirState &s, cudaStream_t stream, KvJob job, int64_t payload_bytes)
 {
     const bool timed = (p->cfg.flags & KV_FLAG_TIME_KERNELS) && s.kev_used < KV_MAX_TIMED;
     if (timed) {
+        if (!s.ktime_dev) {
+            // allocated and preset once; kv_sync presets the slots again after reading them
+            cudaError_t rc = cudaMalloc((void **)&s.ktime_dev, (size_t)KV_MAX_TIMED * 2 * sizeof(unsigned long long));
+            if (rc != cudaSuccess) return rc;
+            rc = preset_ktime(s, stream);
+            if (rc == cudaSuccess) rc = cudaStreamSynchronize(stream);   // once: later launches may come from another stream
+            if (rc != cudaSuccess) return rc;
+        }
+        job.t_first = s.ktime_dev + 2 * (size_t)s.kev_used;
+        job.t_last = job.t_first + 1;
         while ((int)s.kev.size() < 2 * (s.kev_used + 1)) {
             cudaEvent_t e;
             cudaError_t rc = cudaEventCreate(&e);
@@ -955,6 +976,7 @@ int32_t kv_pool_destroy(kv_pool_t *p)
         }
         if (s.kfork_ev) (void)cudaEventDestroy(s.kfork_ev);
         for (cudaEvent_t e : s.kev) (void)cudaEventDestroy(e);
+        if (s.ktime_dev) (void)cudaFree(s.ktime_dev);
         for (int k = 0; k < 2; ++k) {
             if (s.ev_a[k]) (void)cudaEventDestroy(s.ev_a[k]);
             if (s.ev_b[k]) (void)cudaEventDestroy(s.ev_b[k]);
@@ -1165,6 +1187,15 @@ int32_t kv_sync(kv_pool_t *p)
     }
     for (int d = 0; d < 2; ++d) {
         DirState &s = p->dir[d];
+        if (s.kev_used > 0 && s.ktime_dev) {
+            std::vector<unsigned long long> t((size_t)2 * s.kev_used);
+            if (cudaMemcpy(t.data(), s.ktime_dev, t.size() * sizeof(unsigned long long), cudaMemcpyDeviceToHost) == cudaSuccess) {
+                for (int k = 0; k < s.kev_used; ++k)
+                    if (t[2 * (size_t)k + 1] > t[2 * (size_t)k]) p->stats.timed_kernel_exec_ms += (double)(t[2 * (size_t)k + 1] - t[2 * (size_t)k]) * 1e-6;
+                (void)preset_ktime(s, s.kstream);
+                (void)cudaStreamSynchronize(s.kstream);
+            }
+        }
         for (int k = 0; k < s.kev_used; ++k) {
             float ms = 0.f;
             if (cudaEventElapsedTime(&ms, s.kev[2 * (size_t)k], s.kev[2 * (size_t)k + 1]) == cudaSuccess) {
@@ -1514,6 +1545,7 @@ extern "C" int32_t kv_gather_blocks_static(const void *device_base, int32_t num_
     job.chunk = (int)std::min<int64_t>(seg, BULK_STAGE);
     job.cps = (int)((seg + job.chunk - 1) / job.chunk);
     job.status = status;
+    job.t_first = job.t_last = nullptr;
     job.dir[1] = KvDir{};
     KvDir &kd = job.dir[0];
     kd.src = KvSide{(unsigned long long)device_base, seg, num_gpu_blocks * seg};

@@ -47,6 +47,9 @@ struct KvJob {
     int chunk;           // bytes per work item (last chunk of a plane may be shorter)
     int cps;             // chunks per plane
     unsigned int *status;
+    // optional: device words that receive the earliest start and the latest end of the launch's CTAs
+    // (%globaltimer, ns); nullptr = not wanted.  The host presets them to ~0 and 0.
+    unsigned long long *t_first, *t_last;
 };
 
 // ------------------------------------------------------------------------------------------------
@@ -198,6 +201,7 @@ __global__ void __launch_bounds__(32, 1) kv_copy_bulk(const __grid_constant__ Kv
     if (!kv_my_range(job, dsel, lo, hi)) return;
     const KvDir &d = job.dir[dsel];
     constexpr unsigned long long LIMIT_NS = 2000000000ull;   // 2 s per wait
+    if (job.t_first) atomicMin(job.t_first, kv_globaltimer());
 
     const uint32_t smem0 = kv_smem_u32(kv_smem);
     const uint32_t bar0 = kv_smem_u32(full_bar);
@@ -243,6 +247,7 @@ __global__ void __launch_bounds__(32, 1) kv_copy_bulk(const __grid_constant__ Kv
             kv_mbar_wait(bar0 + 8 * (int)(j % NS), (uint32_t)((j / NS) & 1), LIMIT_NS);
     }
     kv_bulk_wait_all();
+    if (job.t_last) atomicMax(job.t_last, kv_globaltimer());
 }
 
 // ------------------------------------------------------------------------------------------------
