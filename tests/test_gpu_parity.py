@@ -141,11 +141,12 @@ def test_config5_replay_scaled():
         p.close()
 
 
-def test_back_to_back_calls_with_cross_direction_dependencies():
+@pytest.mark.parametrize("path", ["zerocopy", "staged", "auto"])
+def test_back_to_back_calls_with_cross_direction_dependencies(path):
     """swap_out(g->h) immediately followed by swap_in(h->g2) with no sync: the library must order the
     second after the first (the host block is written, then read).  Then the reverse dependency."""
     shape = W.KVShape(4, 16, 8, 128)
-    p = _pair(shape, 64, 64, seed=5, path=1)
+    p = _pair(shape, 64, 64, seed=5, path={"auto": 0, **PATHS}[path])
     rng = np.random.default_rng(0)
     try:
         for _ in range(6):
@@ -161,7 +162,7 @@ def test_back_to_back_calls_with_cross_direction_dependencies():
         p.close()
 
 
-@pytest.mark.parametrize("path", ["zerocopy", "ce2d"])
+@pytest.mark.parametrize("path", ["zerocopy", "staged", "ce2d"])
 def test_overlapping_rotate_needs_flag_and_matches_sequential_semantics(path):
     shape = W.KVShape(2, 16, 8, 128)
     rng = np.random.default_rng(2)
