@@ -154,6 +154,32 @@ def time_oracle(shape: W.KVShape, rot: W.Rotation, max_blocks: int, threads: int
     return nbytes, times, f"first {len(og)} out + {len(ig)} in blocks of the rotation ({nbytes / 1e9:.2f} GB per step)"
 
 
+def overlap_of(windows) -> dict:
+    """How much of each timed step had both directions in flight, from the library's per-direction
+    start / end events (swap-out window [0, out], swap-in window [off, off + in])."""
+    fr = []
+    for out_ms, off, in_ms in windows:
+        lo, hi = max(0.0, off), min(out_ms, off + in_ms)
+        union = max(out_ms, off + in_ms) - min(0.0, off)
+        fr.append(max(0.0, hi - lo) / union if union > 0 else 0.0)
+    return {"both_in_flight_share_of_step": float(np.mean(fr)), "min": float(np.min(fr)), "max": float(np.max(fr)),
+            "source": "per-direction start/end events on the library's streams (no nsys on the image)"}
+
+
+def write_trace(path: str, windows) -> None:
+    """Chrome-trace (about://tracing, Perfetto) file of the timed steps: one track per direction."""
+    ev, t = [], 0.0
+    for k, (out_ms, off, in_ms) in enumerate(windows):
+        base = t - min(0.0, off) * 1e3
+        ev.append({"name": f"swap-out step {k}", "ph": "X", "pid": 0, "tid": 0, "ts": base, "dur": out_ms * 1e3})
+        ev.append({"name": f"swap-in step {k}", "ph": "X", "pid": 0, "tid": 1, "ts": base + off * 1e3, "dur": in_ms * 1e3})
+        t = base + max(out_ms, off + in_ms) * 1e3 + 50.0
+    meta = [{"name": "thread_name", "ph": "M", "pid": 0, "tid": 0, "args": {"name": "device to host (swap-out stream)"}},
+            {"name": "thread_name", "ph": "M", "pid": 0, "tid": 1, "args": {"name": "host to device (swap-in stream)"}}]
+    with open(path, "w") as f:
+        json.dump({"traceEvents": meta + ev, "displayTimeUnit": "ms"}, f)
+
+
 # ------------------------------------------------------------------------------------------------ arms
 
 def run_reference(args, rank: int) -> None:
@@ -248,11 +274,13 @@ def run_ours(args, rank: int, local_rank: int, world: int) -> None:
     sampler = ClockSampler(local_rank)
     sampler.start()
     barrier()
-    dev_ms = []
+    dev_ms, windows = [], []
     t0 = time.perf_counter()
     for _ in range(args.steps):
         step()
-        dev_ms.append(pool.kv_get_stats()["last_union_ms"])
+        s_ = pool.kv_get_stats()
+        dev_ms.append(s_["last_union_ms"])
+        windows.append((s_["last_out_ms"], s_["last_in_offset_ms"], s_["last_in_ms"]))
     barrier()
     wall_s = time.perf_counter() - t0
     clocks = sampler.stop()
@@ -264,6 +292,8 @@ def run_ours(args, rank: int, local_rank: int, world: int) -> None:
     k_n = st["timed_kernels"] - st0["timed_kernels"]
     k_exec_ms = st["timed_kernel_exec_ms"] - st0["timed_kernel_exec_ms"]
 
+    if args.trace and rank == 0:
+        write_trace(args.trace, windows)
     dev_total_ms = reduce(float(np.sum(dev_ms)), "max")
     wall_total_s = reduce(wall_s, "max")
     job_bytes = reduce(float(bytes_out + bytes_in), "sum") * args.steps
@@ -429,6 +459,7 @@ def run_ours(args, rank: int, local_rank: int, world: int) -> None:
             "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": bytes_in + 8 * (rot.n_out + rot.n_in),
                     "d2h_bytes_per_step": bytes_out, "ms_per_step": wall_total_s * 1e3 / args.steps},
             "gpu_launches": int(launches), "ce_transfers": int(ce_copies),
+            "overlap": overlap_of(windows),
             "clocks": clocks,
             "roofline": roofline,
             "roofline_link": link,
@@ -471,6 +502,7 @@ def main() -> None:
     ap.add_argument("--ctas", type=int, default=0, help="CTAs per direction (0 = default)")
     ap.add_argument("--staging-mib", type=int, default=0, help="per-direction staging of the staged path (0 = library default)")
     ap.add_argument("--quick", action="store_true", help="skip the per-segment comparator path")
+    ap.add_argument("--trace", default=None, help="write a Chrome-trace JSON of the timed steps' two directions here")
     ap.add_argument("--small", action="store_true",
                     help="profiling case: same shape and kernels, 16 requests, 4 rotated each way, 6 GB + 8 GB pools")
     args = ap.parse_args()

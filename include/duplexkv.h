@@ -125,6 +125,8 @@ typedef struct {
     int64_t timed_kernels;             /* how many launches the two sums cover                            */
     double  timed_kernel_exec_ms;      /* the same launches timed from inside: earliest CTA start to latest
                                           CTA end (%globaltimer), i.e. without the wait for the launch     */
+    double  last_in_offset_ms;         /* latest kv_rotate: start of its swap-in window minus start of its
+                                          swap-out window (with last_out_ms and last_in_ms: the timeline)  */
 } kv_stats_t;
 
 typedef struct {

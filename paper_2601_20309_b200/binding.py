@@ -60,7 +60,7 @@ class kv_stats_t(C.Structure):
                 ("last_path_out", C.c_int32), ("last_path_in", C.c_int32),
                 ("device_status", C.c_uint32), ("pad_", C.c_int32),
                 ("timed_kernel_ms", C.c_double), ("timed_kernel_bytes", C.c_int64), ("timed_kernels", C.c_int64),
-                ("timed_kernel_exec_ms", C.c_double)]
+                ("timed_kernel_exec_ms", C.c_double), ("last_in_offset_ms", C.c_double)]
 
 
 class kv_link_probe_t(C.Structure):

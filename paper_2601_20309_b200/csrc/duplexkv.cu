@@ -1179,8 +1179,10 @@ int32_t kv_sync(kv_pool_t *p)
             off = (fwd && a > 0.f) ? a : ((bwd && b > 0.f) ? -b : 0.f);
             const float lo = std::min(0.f, off), hi = std::max(t_out, off + t_in);
             p->stats.last_union_ms = hi - lo;
+            p->stats.last_in_offset_ms = off;
         } else {
             p->stats.last_union_ms = so >= 0 ? t_out : t_in;
+            p->stats.last_in_offset_ms = 0.0;
         }
         (void)cudaGetLastError();
         p->union_valid = false;

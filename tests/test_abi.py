@@ -43,6 +43,6 @@ def test_shape_helpers_need_no_device():
 def test_struct_sizes_match_the_header_layout():
     # natural alignment on both sides; a mismatch here means the ctypes mirror drifted from the header
     assert C.sizeof(B.kv_pool_config_t) == 112
-    assert C.sizeof(B.kv_stats_t) == 120
+    assert C.sizeof(B.kv_stats_t) == 128
     assert C.sizeof(B.kv_link_probe_t) == 56
     assert C.sizeof(B.kv_probe_spec_t) == 56
