@@ -404,8 +404,8 @@ def run_ours(args, rank: int, local_rank: int, world: int) -> None:
     if rank == 0:
         # ---- CPU oracle on the host cores, bounded sample of the same rotation
         threads = os.cpu_count() or 1
-        nb_s, t_mt, sample = time_oracle(shape, rot, 768, threads, reps=3)
-        _, t_1, _ = time_oracle(shape, rot, 256, 1, reps=2)
+        nb_s, t_mt, sample = time_oracle(shape, rot, 768, threads, reps=20, warmup=2)
+        _, t_1, _ = time_oracle(shape, rot, 256, 1, reps=5)
         cpu_val = M.gbs(nb_s, float(np.mean(t_mt)) * 1e3)
         cpu_1 = M.gbs(2 * 256 * shape.block_bytes, float(np.mean(t_1)) * 1e3)
 
