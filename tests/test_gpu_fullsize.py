@@ -170,3 +170,26 @@ def test_config5_full_shape_replay_2000_steps():
         t.verify("config 5 replay")
     finally:
         t.close()
+
+
+@pytest.mark.parametrize("bs,contiguous,payload", [(8, False, 2e9), (64, True, 4e9), (32, False, 4e9)],
+                         ids=["block8-random-2GB", "block64-contiguous-4GB", "block32-random-4GB"])
+def test_config4_sweep_cells_at_full_payload(bs, contiguous, payload):
+    """Cells of the block-size / fragmentation sweep at full payload, default path: 1 MiB blocks with random
+    tables (the zero-copy kernels), 8 MiB blocks with contiguous tables (long merged transfers), 4 MiB
+    blocks with random tables (uniform two-block transfers).  Each direction alone, then both at once."""
+    w = W.config4_sweep_case(bs, contiguous, payload)
+    t = _FullSize(w)
+    try:
+        r = w.steps[0]
+        t.swap_out(r.out_gpu, r.out_host)
+        moved = t.verify("swap-out alone", n_read_back=4)
+        assert moved == (0, r.n_out)
+        t.swap_in(r.in_host, r.in_gpu)
+        t.rotate(r)
+        moved = t.verify("swap-in alone, then both at once", n_read_back=4)
+        assert moved == (r.n_in, r.n_out)
+        want = "zerocopy" if bs == 8 and not contiguous else "staged"
+        assert t.B.PATH_NAMES[t.pool.kv_get_stats()["last_path_out"]] == want
+    finally:
+        t.close()
