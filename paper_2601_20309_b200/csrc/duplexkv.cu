@@ -334,6 +334,8 @@ struct DirCall {
     // copy-engine issue state (CE paths are issued in slices so the two directions interleave)
     int64_t ce_next = 0;
     bool planned = false;              // STAGED: plan_staged has run for this call
+    int64_t plan_nruns = 0;            //         runs of consecutive host ids in its list
+    bool plan_uniform = false;         //         the plan uses uniform two-block transfers
     int chunk_idx = 0;                 // STAGED: chunk being issued, next op of it
     int op_next = 0;
     bool chunk_open = false;
@@ -375,8 +377,11 @@ struct PlanParams {
 
 // Pure planning (no pool, no CUDA): order, transfers and chunks for n pairs of direction d (0 out, 1 in)
 // whose host block ids are host_ids.  May throw std::bad_alloc.
+// mode: -1 = decide from this list's runs, 0 = merge runs, 1 = uniform two-block transfers;
+// *nruns_out / *uniform_out (may be null) report the list's runs of consecutive host ids and the mode taken.
 void plan_transfers(const PlanParams &pp, int d, const int32_t *host_ids, int64_t n, std::vector<int32_t> &order,
-                    std::vector<CeOp> &ops, std::vector<CeChunk> &chunks)
+                    std::vector<CeOp> &ops, std::vector<CeChunk> &chunks, int mode = -1, int64_t *nruns_out = nullptr,
+                    bool *uniform_out = nullptr)
 {
     {
         order.resize((size_t)n);
@@ -415,7 +420,9 @@ void plan_transfers(const PlanParams &pp, int d, const int32_t *host_ids, int64_
         int64_t nruns = 1;
         for (int64_t q = 1; q < n; ++q)
             if (hid(q) != hid(q - 1) + 1) ++nruns;
-        const bool uniform = n < KV_MERGE_MIN_MEAN_RUN * nruns;
+        const bool uniform = mode < 0 ? n < KV_MERGE_MIN_MEAN_RUN * nruns : mode == 1;
+        if (nruns_out) *nruns_out = nruns;
+        if (uniform_out) *uniform_out = uniform;
         auto run_len = [&](int64_t q) {
             int64_t r = 1;
             if (uniform) return r;
@@ -461,13 +468,13 @@ void plan_transfers(const PlanParams &pp, int d, const int32_t *host_ids, int64_
     }
 }
 
-int32_t plan_staged(kv_pool *p, DirCall &c)
+int32_t plan_staged(kv_pool *p, DirCall &c, int mode = -1)
 {
     DirState &s = p->dir[c.d];
     const PlanParams pp{p->blk, p->seg, s.half_blocks, p->max_pitch, p->cfg.num_host_blocks, p->planes,
                         p->cfg.host_layout == KV_HOST_LAYER_FIRST};
     try {
-        plan_transfers(pp, c.d, c.host_ids, c.n, s.order, s.ops, s.chunks);
+        plan_transfers(pp, c.d, c.host_ids, c.n, s.order, s.ops, s.chunks, mode, &c.plan_nruns, &c.plan_uniform);
     } catch (...) {
         return fail(p, KV_ERR_NOMEM, "out of host memory");
     }
@@ -745,6 +752,24 @@ int32_t run_calls(kv_pool *p, DirCall *calls, int ncalls, const bool *wait_other
         const int chosen = (ops > 0 && bytes >= ops * KV_AUTO_MIN_TRANSFER) ? KV_PATH_STAGED : KV_PATH_ZEROCOPY;
         for (int k = 0; k < ncalls; ++k)
             if (calls[k].path == KV_PATH_AUTO) calls[k].path = chosen;
+    }
+    // Both directions of a staged rotate use the same kind of transfers: two-block transfers one way and
+    // long merged ones the other way fall out of step (74 GB/s measured against 88 to 95 when alike).
+    if (ncalls == 2 && calls[0].path == KV_PATH_STAGED && calls[1].path == KV_PATH_STAGED &&
+        p->cfg.host_layout == KV_HOST_BLOCK_FIRST) {
+        for (int k = 0; k < 2; ++k)
+            if (!calls[k].planned) {
+                int32_t rc = plan_staged(p, calls[k]);
+                if (rc != KV_OK) return rc;
+            }
+        if (calls[0].plan_uniform != calls[1].plan_uniform) {
+            const bool joint = calls[0].n + calls[1].n < KV_MERGE_MIN_MEAN_RUN * (calls[0].plan_nruns + calls[1].plan_nruns);
+            for (int k = 0; k < 2; ++k)
+                if (calls[k].plan_uniform != joint) {
+                    int32_t rc = plan_staged(p, calls[k], joint ? 1 : 0);
+                    if (rc != KV_OK) return rc;
+                }
+        }
     }
     for (int k = 0; k < ncalls; ++k) {
         if (fused && calls[k].d == 1) {

@@ -313,6 +313,16 @@ def test_staged_transfer_planning_patterns(layout):
             ih = rng.choice(np.setdiff1d(np.arange(nbh), oh), 40, replace=False).astype(np.int32)
             assert p.rotate_both(W.Rotation(og, oh, ih, ig, np.zeros(1), np.zeros(1))) == 0
         p.assert_equal("staged rotate, queued")
+        # one direction with a long run of host ids, the other scattered: both must end up on the same kind
+        # of transfers (the plan of one of them is redone), whichever direction has the run
+        for flip in (False, True):
+            og = rng.choice(nbg, 40, replace=False).astype(np.int32)
+            ig = np.setdiff1d(np.arange(nbg), og)[:40].astype(np.int32)
+            run = np.arange(150, 190, dtype=np.int32)
+            scattered = rng.choice(np.setdiff1d(np.arange(nbh), run), 40, replace=False).astype(np.int32)
+            oh, ih = (scattered, run) if flip else (run, scattered)
+            assert p.rotate_both(W.Rotation(og, oh, ih, ig, np.zeros(1), np.zeros(1))) == 0
+            p.assert_equal(f"staged rotate, mixed host id patterns, flip={flip}")
         st = p.pool.kv_get_stats()
         assert st["device_status"] == 0 and st["kernel_launches"] > 0
     finally:
