@@ -31,7 +31,11 @@ class Pair:
             for pl in range(2 * s.num_layers):
                 off = o.host_off(h, pl // 2, pl % 2) // 2
                 H16[off:off + wpp] = words[pl]
-        self.dev = torch.from_numpy(o.G.copy()).to("cuda:0")
+        # the device pool sits between two guard areas of one block each, which no call may touch
+        self.guard = -(-max(256, s.block_bytes) // 256) * 256
+        self.buf = torch.full((o.G.size + 2 * self.guard,), 0xC3, dtype=torch.uint8, device="cuda:0")
+        self.dev = self.buf[self.guard:self.guard + o.G.size]
+        self.dev.copy_(torch.from_numpy(o.G))
         self.pool = B.KVPool(s.num_layers, s.block_size, s.kv_heads, s.head_dim, nb_gpu, nb_host,
                              self.dev.data_ptr(), host_layout=host_layout, device_layout=device_layout, **pool_kw)
         self.pool.host_array()[:] = o.Hs
@@ -44,6 +48,9 @@ class Pair:
         self.pool.kv_sync()
         g = self.gpu_bytes()
         h = self.pool.host_array()
+        lo, hi = self.buf[:self.guard], self.buf[self.guard + g.size:]
+        if not (bool((lo == 0xC3).all()) and bool((hi == 0xC3).all())):
+            raise AssertionError(f"{what}: bytes outside the device pool were written")
         if not np.array_equal(g, self.oracle.G):
             bad = np.flatnonzero(g != self.oracle.G)
             raise AssertionError(f"{what}: device pool differs at {len(bad)} bytes, first {bad[:4]}")
