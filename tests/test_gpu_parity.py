@@ -419,3 +419,45 @@ def test_budgeted_replay_matches_the_oracle():
         p.assert_equal("budgeted replay")
     finally:
         p.close()
+
+
+@pytest.mark.parametrize("path", ["zerocopy", "staged"])
+def test_caller_supplied_host_memory_is_page_locked_and_stays_inside_its_bounds(path):
+    """host_base given by the caller: the library page-locks it for the pool's lifetime, moves the same
+    bytes as with its own allocation, and writes nothing outside the region it was given."""
+    import torch
+    from oracle.kv_oracle import ByteOracle
+    from paper_2601_20309_b200 import binding as B
+    shape = W.KVShape(3, 16, 8, 128)
+    nbg, nbh = 40, 60
+    o = ByteOracle(shape.num_layers, shape.block_size, shape.kv_heads, shape.head_dim, nbg, nbh)
+    rng = np.random.default_rng(31)
+    o.G[:] = rng.integers(0, 256, o.G.size, dtype=np.uint8)
+    o.Hs[:] = rng.integers(0, 256, o.Hs.size, dtype=np.uint8)
+    page, size = 4096, nbh * shape.block_bytes
+    raw = np.full(size + 3 * page, 0x5A, np.uint8)
+    start = (-raw.ctypes.data) % page + page                    # page-aligned, one guard page before
+    region = raw[start:start + size]
+    region[:] = o.Hs
+    dev = torch.from_numpy(o.G.copy()).to("cuda:0")
+    pool = B.KVPool(shape.num_layers, shape.block_size, shape.kv_heads, shape.head_dim, nbg, nbh, dev.data_ptr(),
+                    host_base=region.ctypes.data, path=PATHS[path])
+    try:
+        base, nbytes = pool.kv_host_ptr()
+        assert base == region.ctypes.data and nbytes == size
+        og = rng.choice(nbg, 15, replace=False).astype(np.int32)
+        ig = np.setdiff1d(np.arange(nbg), og)[:12].astype(np.int32)
+        oh = rng.choice(nbh, 15, replace=False).astype(np.int32)
+        ih = rng.choice(np.setdiff1d(np.arange(nbh), oh), 12, replace=False).astype(np.int32)
+        assert o.rotate(og, oh, ih, ig) == 0 and pool.kv_rotate(og, oh, ih, ig) == 0
+        pool.kv_sync()
+        assert np.array_equal(region, o.Hs)
+        assert np.array_equal(dev.cpu().numpy(), o.G)
+        assert (raw[:start] == 0x5A).all() and (raw[start + size:] == 0x5A).all()
+    finally:
+        pool.destroy()
+    region[:8] = 1                                                # still ordinary memory after the pool is gone
+    # a misaligned host_base is refused
+    with pytest.raises(B.KVError):
+        B.KVPool(shape.num_layers, shape.block_size, shape.kv_heads, shape.head_dim, nbg, nbh, dev.data_ptr(),
+                 host_base=region.ctypes.data + 8)
