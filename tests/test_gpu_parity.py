@@ -461,3 +461,51 @@ def test_caller_supplied_host_memory_is_page_locked_and_stays_inside_its_bounds(
     with pytest.raises(B.KVError):
         B.KVPool(shape.num_layers, shape.block_size, shape.kv_heads, shape.head_dim, nbg, nbh, dev.data_ptr(),
                  host_base=region.ctypes.data + 8)
+
+
+@pytest.mark.parametrize("knobs", [
+    dict(path=1, path_in=2), dict(path=2, path_in=1), dict(path=3, path_in=1), dict(path=3, ce_streams=4),
+    dict(path=4, ce_streams=2), dict(path=1, ctas_out=3, ctas_in=148), dict(path=1, flags=4, ctas_out=5, ctas_in=9),
+    dict(path=2, staging_bytes=1), dict(path=0, flags=8),
+], ids=lambda k: "-".join(f"{a}{b}" for a, b in k.items()))
+def test_tuning_knobs_do_not_change_results(knobs):
+    """A different path per direction, several copy-engine streams, odd CTA counts, the smallest staging,
+    kernel timing: every setting must give the oracle's bytes."""
+    w = W.config2_8b(nb_gpu=320, nb_host=448, n_req=16, median=96, max_tokens=512, n_rot=4)
+    p = _pair(w.shape, w.nb_gpu, w.nb_host, seed=w.seed, **knobs)
+    try:
+        assert p.rotate_both(w.steps[0]) == 0
+        for r in w.extra["pairs"][:4]:
+            assert p.rotate_both(r) == 0
+        p.assert_equal(f"knobs {knobs}")
+        assert p.pool.kv_get_stats()["device_status"] == 0
+    finally:
+        p.close()
+
+
+def test_caller_streams_and_link_probe():
+    """Streams made by the caller (here: torch) carry the two directions; and the link probe returns
+    sensible figures for plain and strided transfers and refuses nonsense."""
+    import torch
+    from paper_2601_20309_b200 import binding as B
+    s_out, s_in = torch.cuda.Stream(), torch.cuda.Stream()
+    w = W.config1_tiny()
+    p = _pair(w.shape, w.nb_gpu, w.nb_host, seed=w.seed, stream_out=s_out.cuda_stream, stream_in=s_in.cuda_stream, path=2)
+    try:
+        assert p.rotate_both(w.steps[0]) == 0
+        s_out.synchronize()
+        s_in.synchronize()                             # the caller's own streams are what the work ran on
+        assert np.array_equal(p.pool.host_array(), p.oracle.Hs)
+        p.assert_equal("caller streams")
+        assert p.pool.kv_pool_progress() == {"out_issued": 1, "out_done": 1, "in_issued": 1, "in_done": 1}
+    finally:
+        p.close()
+    plain = B.kv_probe_link_ex(0, copy_bytes=1 << 20, total_bytes=32 << 20, span_bytes=64 << 20, scattered=True, rounds=1)
+    strided = B.kv_probe_link_ex(0, copy_bytes=2 << 20, total_bytes=32 << 20, span_bytes=64 << 20, scattered=True, rounds=1,
+                                 rows=2, host_pitch=8 << 20)
+    for r in (plain, strided):
+        assert 1.0 < r["d2h_gbs"] < 200.0 and 1.0 < r["h2d_gbs"] < 200.0 and r["bi_sum_gbs"] > r["d2h_gbs"] * 0.8
+    with pytest.raises(B.KVError):
+        B.kv_probe_link_ex(0, copy_bytes=3 << 20, total_bytes=32 << 20, span_bytes=64 << 20, rows=2, host_pitch=1 << 20)
+    with pytest.raises(B.KVError):
+        B.kv_probe_link_ex(0, copy_bytes=1 << 20, total_bytes=1 << 10, span_bytes=64 << 20)
