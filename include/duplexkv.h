@@ -202,6 +202,18 @@ int32_t kv_plan_staged(int64_t blk_bytes, int64_t half_blocks, int32_t direction
  * re-applies the rule of kv_path_for).  Pool contents are unaffected. */
 int32_t kv_pool_set_path(kv_pool_t *pool, int32_t path_out, int32_t path_in);
 
+/*
+ * Bound of the waits inside the copy kernels (each wait of a kernel's main loop for a load it has
+ * issued): `polls` immediate polls, then polls 200 ns apart for at most `ns` nanoseconds (default 16 and
+ * 2 s; ns <= 60 s).  A wait that runs out makes its CTA record KV_DEV_TIMEOUT in the pool's status word,
+ * wait (with the default bound) for the loads it still has in flight, drain its stores and return; the
+ * bytes it had left are not moved, kv_sync reports KV_ERR_TIMEOUT and the pool stays in that state.
+ * polls == 0 and ns == 0 make every such wait give up without looking, which is how the failure path is
+ * exercised on a healthy GPU without a fault or a hang.  Applies to calls issued afterwards.  (Failure
+ * handling of this library; the paper describes none.)
+ */
+int32_t kv_pool_set_wait_limit(kv_pool_t *pool, uint32_t polls, uint64_t ns);
+
 /* Wait for both directions.  Returns KV_OK, or the first sticky asynchronous error
  * (KV_ERR_CUDA, KV_ERR_TIMEOUT).  Fills the last_* timing fields of the statistics. */
 int32_t kv_sync(kv_pool_t *pool);
@@ -210,7 +222,11 @@ int32_t kv_sync(kv_pool_t *pool);
  * Device-side gather / scatter (the kernel half of the STAGED path, also usable on its own):
  * gather copies the listed device blocks, in list order, into a contiguous DEVICE buffer laid out
  * block-first (block i at i*BLK, planes in (layer, K|V) order); scatter is the inverse.  dst/src must
- * hold n*BLK bytes and be 16-byte aligned.  Runs on the out (gather) / in (scatter) stream.
+ * hold n*BLK bytes and be 16-byte aligned.  Runs on the out (gather) / in (scatter) stream and is
+ * ordered like a call of that direction: a gather waits for an unfinished swap-in (or scatter) that
+ * writes one of its blocks, a scatter for an unfinished swap-out (or gather) that reads one of its
+ * blocks, and later calls of the other direction wait for it in the same way.  The buffer itself is
+ * the caller's: nothing orders other work on dst_device / src_device.
  * This is the "merge small segments into large contiguous regions" step of section 4.3, done by
  * a kernel instead of a layout change.
  */
@@ -376,11 +392,12 @@ int32_t kv_req_add(kv_table_t *table, int64_t req, int64_t tokens);
 int32_t kv_req_append(kv_table_t *table, int64_t req, int64_t new_tokens);
 /* Background step: copy up to max_blocks full blocks that have no valid host copy to host memory
  * (requests in arrival order, round robin across calls) with one kv_swap_out, and mark them synced.
- * *n_issued (may be NULL) = blocks sent.  Sends fewer when the host pool runs out. */
+ * *n_issued (may be NULL) = blocks sent.  Sends fewer when the host pool runs out.  If the pool refuses
+ * the copy, the pool's status is returned and the table is as it was before the call. */
 int32_t kv_eager_rotate(kv_table_t *table, int64_t max_blocks, int64_t *n_issued);
 /* Preempt the listed requests (HOST array of ids; must be on the GPU) and resume the listed ones
- * (must be preempted) in one full-duplex kv_rotate.  All or nothing: KV_ERR_NOMEM / KV_ERR_INVALID_ARG
- * leave the table unchanged. */
+ * (must be preempted) in one full-duplex kv_rotate.  All or nothing: KV_ERR_NOMEM / KV_ERR_INVALID_ARG,
+ * and any status with which the pool refuses the rotation, leave the table unchanged. */
 int32_t kv_req_rotate(kv_table_t *table, const int64_t *preempt, int64_t n_preempt,
                       const int64_t *resume, int64_t n_resume);
 int32_t kv_req_preempt(kv_table_t *table, int64_t req);
@@ -394,6 +411,12 @@ int32_t kv_req_info(kv_table_t *table, int64_t req, kv_req_info_t *out);
 int32_t kv_req_blocks(kv_table_t *table, int64_t req, int32_t *gpu_ids, int32_t *host_ids,
                       uint8_t *host_valid, int64_t cap);
 int32_t kv_table_get_stats(kv_table_t *table, kv_table_stats_t *out);
+/* Fault injection for tests, on the host only: the pool call the table makes after `after_calls` further
+ * ones (0 = the very next kv_swap_out / kv_rotate it would issue) is not made and counts as having
+ * returned `code` (a negative KV_ERR_*); later calls go through again.  after_calls < 0 disarms.  Works on
+ * a dry table too.  Nothing is sent to the device, so no transfer is ever half done.  (The paper has no
+ * counterpart; this is how the all-or-nothing promise of kv_req_rotate and kv_eager_rotate is tested.) */
+int32_t kv_table_fail_pool_call(kv_table_t *table, int64_t after_calls, int32_t code);
 
 #ifdef __cplusplus
 }

@@ -104,7 +104,8 @@ EXPORTS = ["kv_pool_create", "kv_pool_destroy", "kv_pool_set_path", "kv_swap_out
            "kv_gather_blocks_static", "kv_pool_shape", "kv_pool_progress", "kv_stream_wait", "kv_plan_staged",
            "kv_table_create", "kv_table_create_dry", "kv_table_destroy", "kv_table_last_error", "kv_req_add",
            "kv_req_append", "kv_eager_rotate", "kv_req_rotate", "kv_req_preempt", "kv_req_resume", "kv_req_finish",
-           "kv_req_info", "kv_req_blocks", "kv_table_get_stats"]
+           "kv_req_info", "kv_req_blocks", "kv_table_get_stats", "kv_table_fail_pool_call",
+           "kv_pool_set_wait_limit"]
 
 _lib = None
 
@@ -183,6 +184,10 @@ def lib() -> C.CDLL:
     L.kv_req_blocks.argtypes = [vp, i64, i32p, i32p, C.POINTER(C.c_uint8), i64]
     L.kv_table_get_stats.restype = C.c_int32
     L.kv_table_get_stats.argtypes = [vp, C.POINTER(kv_table_stats_t)]
+    L.kv_pool_set_wait_limit.restype = C.c_int32
+    L.kv_pool_set_wait_limit.argtypes = [vp, C.c_uint32, C.c_uint64]
+    L.kv_table_fail_pool_call.restype = C.c_int32
+    L.kv_table_fail_pool_call.argtypes = [vp, i64, C.c_int32]
     L.kv_gather_blocks_static.restype = C.c_int32
     L.kv_gather_blocks_static.argtypes = [vp, C.c_int32, C.c_int32, C.c_int32, C.c_int32, i64, i32p, i64, vp, vp]
     L.kv_probe_link_ex.restype = C.c_int32
@@ -344,6 +349,9 @@ class KVPool:
     def kv_pool_set_path(self, path_out: int, path_in: int, check: bool = True) -> int:
         return self._ret(lib().kv_pool_set_path(self._h, path_out, path_in), check)
 
+    def kv_pool_set_wait_limit(self, polls: int, ns: int, check: bool = True) -> int:
+        return self._ret(lib().kv_pool_set_wait_limit(self._h, polls, ns), check)
+
     def kv_sync(self, check: bool = True) -> int:
         return self._ret(lib().kv_sync(self._h), check)
 
@@ -458,6 +466,9 @@ class KVTable:
         self._ret(lib().kv_req_blocks(self._h, req, g.ctypes.data_as(i32p), h.ctypes.data_as(i32p),
                                       v.ctypes.data_as(C.POINTER(C.c_uint8)), n), True)
         return g, h, v.astype(bool)
+
+    def kv_table_fail_pool_call(self, after_calls: int, code: int) -> int:
+        return self._ret(lib().kv_table_fail_pool_call(self._h, after_calls, code), True)
 
     def kv_table_get_stats(self) -> dict:
         out = kv_table_stats_t()

@@ -41,7 +41,7 @@ def build(force: bool = False, verbose: bool = False) -> str:
     jobs = [(LIB, main_src, main_dep)]
     util_src = os.path.join(CSRC, "kv_testutil.cu")
     if os.path.exists(util_src):
-        jobs.append((TESTUTIL_LIB, [util_src], []))
+        jobs.append((TESTUTIL_LIB, [util_src], [os.path.join(CSRC, "kv_kernels.cuh")]))
     for target, sources, deps in jobs:
         if not force and not _stale(target, sources + deps):
             continue

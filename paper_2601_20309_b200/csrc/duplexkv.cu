@@ -108,6 +108,8 @@ struct kv_pool {
     bool union_valid = false;
     int union_slot[2] = {-1, -1};      // slots of the latest call (per direction; -1 = not part of it)
     int32_t sticky = KV_OK;
+    unsigned int wait_polls = KV_WAIT_POLLS;            // bound of the kernels' main-loop waits (kv_pool_set_wait_limit)
+    unsigned long long wait_ns = KV_WAIT_NS;
     char err[256];
 };
 
@@ -175,6 +177,8 @@ void fill_geometry(const kv_pool *p, KvJob &job, bool link = false)
     job.chunk = (int)std::min<int64_t>(p->seg, max_chunk);
     job.cps = (int)((p->seg + job.chunk - 1) / job.chunk);
     job.status = p->status_dev;
+    job.wait_polls = p->wait_polls;
+    job.wait_ns = p->wait_ns;
     job.t_first = job.t_last = nullptr;
 }
 
@@ -298,6 +302,7 @@ void poll_done(kv_pool *p)
 }
 
 // does a new call of direction `d` touch a block that an unfinished call of the other direction uses?
+// (host_ids == nullptr: a device-side gather / scatter, which names device blocks only)
 bool conflicts_with_other(kv_pool *p, int d, const int32_t *gpu_ids, const int32_t *host_ids, int64_t n)
 {
     const DirState &o = p->dir[1 - d];
@@ -305,7 +310,7 @@ bool conflicts_with_other(kv_pool *p, int d, const int32_t *gpu_ids, const int32
     const std::vector<uint64_t> &gside = (d == 0) ? p->g_written_by_in : p->g_read_by_out;
     const std::vector<uint64_t> &hside = (d == 0) ? p->h_read_by_in : p->h_written_by_out;
     for (int64_t i = 0; i < n; ++i)
-        if (gside[gpu_ids[i]] > o.done || hside[host_ids[i]] > o.done) return true;
+        if (gside[gpu_ids[i]] > o.done || (host_ids && hside[host_ids[i]] > o.done)) return true;
     return false;
 }
 
@@ -315,7 +320,7 @@ void note_use(kv_pool *p, int d, const int32_t *gpu_ids, const int32_t *host_ids
     std::vector<uint64_t> &hside = (d == 0) ? p->h_written_by_out : p->h_read_by_in;
     for (int64_t i = 0; i < n; ++i) {
         gside[gpu_ids[i]] = seq;
-        hside[host_ids[i]] = seq;
+        if (host_ids) hside[host_ids[i]] = seq;
     }
 }
 
@@ -482,6 +487,25 @@ int32_t plan_staged(kv_pool *p, DirCall &c, int mode = -1)
     return KV_OK;
 }
 
+// Everything about a direction of a call that can be refused for lack of memory (the staging buffer, the
+// transfer plan).  Runs for every direction of a call before any of them is begun, so that a refusal
+// leaves no direction half issued: no sequence number taken, no block marked as in use.
+int32_t prepare_dir(kv_pool *p, DirCall &c)
+{
+    DirState &s = p->dir[c.d];
+    if (c.path != KV_PATH_STAGED) return KV_OK;
+    if (!s.stage) {
+        cudaError_t e = cudaMalloc((void **)&s.stage, (size_t)(2 * s.half_blocks * p->blk));
+        if (e != cudaSuccess) {
+            s.stage = nullptr;
+            (void)cudaGetLastError();
+            return fail(p, KV_ERR_NOMEM, "staging buffer allocation failed");
+        }
+    }
+    if (!c.planned) return plan_staged(p, c);
+    return KV_OK;
+}
+
 // wait_for: end event of the other direction's call this one must follow, or nullptr
 int32_t begin_dir(kv_pool *p, DirCall &c, cudaEvent_t wait_for)
 {
@@ -494,18 +518,6 @@ int32_t begin_dir(kv_pool *p, DirCall &c, cudaEvent_t wait_for)
     c.aux_host = c.pairs_host + p->cap;
     c.aux_dev = c.pairs_dev + p->cap;
     if (c.path == KV_PATH_STAGED) {
-        if (!s.stage) {
-            cudaError_t e = cudaMalloc((void **)&s.stage, (size_t)(2 * s.half_blocks * p->blk));
-            if (e != cudaSuccess) {
-                s.stage = nullptr;
-                (void)cudaGetLastError();
-                return fail(p, KV_ERR_NOMEM, "staging buffer allocation failed");
-            }
-        }
-        if (!c.planned) {
-            int32_t rc = plan_staged(p, c);
-            if (rc != KV_OK) return rc;
-        }
         // the kernel sees (device block id, position in the sorted list)
         for (int64_t k = 0; k < c.n; ++k) {
             const int32_t g = c.gpu_ids[s.order[(size_t)k]];
@@ -770,6 +782,10 @@ int32_t run_calls(kv_pool *p, DirCall *calls, int ncalls, const bool *wait_other
                     if (rc != KV_OK) return rc;
                 }
         }
+    }
+    for (int k = 0; k < ncalls; ++k) {
+        int32_t rc = prepare_dir(p, calls[k]);
+        if (rc != KV_OK) return rc;
     }
     for (int k = 0; k < ncalls; ++k) {
         if (fused && calls[k].d == 1) {
@@ -1181,6 +1197,15 @@ int32_t kv_pool_set_path(kv_pool_t *p, int32_t path_out, int32_t path_in)
     return KV_OK;
 }
 
+int32_t kv_pool_set_wait_limit(kv_pool_t *p, uint32_t polls, uint64_t ns)
+{
+    if (!p) return KV_ERR_INVALID_ARG;
+    if (ns > 60ull * 1000000000ull) return fail(p, KV_ERR_INVALID_ARG, "wait limit beyond 60 s");
+    p->wait_polls = polls;
+    p->wait_ns = ns;
+    return KV_OK;
+}
+
 int32_t kv_sync(kv_pool_t *p)
 {
     if (!p) return KV_ERR_INVALID_ARG;
@@ -1258,12 +1283,22 @@ static int32_t device_leg(kv_pool_t *p, const int32_t *gpu_ids, int64_t n, const
         if (rc != KV_OK) return rc;
     }
     DirState &s = p->dir[d];
+    // Ordered like a swap call of its direction: a gather reads device blocks (as a swap-out does), a
+    // scatter writes them (as a swap-in does), so it waits for an unfinished call of the other direction
+    // that writes / reads one of its blocks, and later calls of the other direction wait for it.
+    poll_done(p);
+    cudaEvent_t wait_for = nullptr;
+    if (conflicts_with_other(p, d, gpu_ids, nullptr, n)) {
+        const DirState &o = p->dir[1 - d];
+        wait_for = o.ev_end[o.issued % KV_SLOTS];
+    }
     const uint64_t seq = s.issued + 1;
     const int slot = (int)(seq % KV_SLOTS);
     if (seq > KV_SLOTS) KV_CUDA(p, cudaEventSynchronize(s.ev_end[slot]));
     int2 *ph = s.ring_host + (size_t)slot * 2 * p->cap;
     int2 *pd = s.ring_dev + (size_t)slot * 2 * p->cap;
     for (int64_t i = 0; i < n; ++i) ph[i] = (d == 0) ? make_int2(gpu_ids[i], (int)i) : make_int2((int)i, gpu_ids[i]);
+    if (wait_for) KV_CUDA(p, cudaStreamWaitEvent(s.stream, wait_for, 0));
     KV_CUDA(p, cudaEventRecord(s.ev_start[slot], s.stream));
     KV_CUDA(p, cudaMemcpyAsync(pd, ph, (size_t)n * sizeof(int2), cudaMemcpyHostToDevice, s.stream));
     KvJob job;
@@ -1279,6 +1314,7 @@ static int32_t device_leg(kv_pool_t *p, const int32_t *gpu_ids, int64_t n, const
     KV_CUDA(p, launch_timed(p, s, s.stream, job, n * p->blk));
     KV_CUDA(p, cudaEventRecord(s.ev_end[slot], s.stream));
     s.issued = seq;
+    note_use(p, d, gpu_ids, nullptr, n, seq);
     p->union_slot[d] = slot;
     p->union_slot[1 - d] = -1;
     p->union_valid = true;
@@ -1572,6 +1608,8 @@ extern "C" int32_t kv_gather_blocks_static(const void *device_base, int32_t num_
     job.chunk = (int)std::min<int64_t>(seg, BULK_STAGE);
     job.cps = (int)((seg + job.chunk - 1) / job.chunk);
     job.status = status;
+    job.wait_polls = KV_WAIT_POLLS;
+    job.wait_ns = KV_WAIT_NS;
     job.t_first = job.t_last = nullptr;
     job.dir[1] = KvDir{};
     KvDir &kd = job.dir[0];

@@ -19,8 +19,9 @@
 //               chunk issued before its stores; each warp walks the pair list cooperatively
 //               (one coalesced load of up to 32 pairs, then shuffles).
 //
-// Every wait on an mbarrier is bounded: when it runs out the thread sets KV_DEV_TIMEOUT in the
-// job's status word, drains what it has in flight and returns.
+// Every wait on an mbarrier is bounded (the job carries the bound of the main-loop waits): when one
+// runs out the thread sets KV_DEV_TIMEOUT in the job's status word, waits -- again bounded -- for the
+// loads it has in flight, drains its stores and returns.
 #pragma once
 #include <cuda_runtime.h>
 #include <stdint.h>
@@ -47,6 +48,10 @@ struct KvJob {
     int chunk;           // bytes per work item (last chunk of a plane may be shorter)
     int cps;             // chunks per plane
     unsigned int *status;
+    // bound of every wait for a load in the kernels' main loops: `wait_polls` immediate polls, then polls
+    // 200 ns apart for at most `wait_ns` nanoseconds (0 = give up right after the immediate polls)
+    unsigned int wait_polls;
+    unsigned long long wait_ns;
     // optional: device words that receive the earliest start and the latest end of the launch's CTAs
     // (%globaltimer, ns); nullptr = not wanted.  The host presets them to ~0 and 0.
     unsigned long long *t_first, *t_last;
@@ -144,14 +149,18 @@ __device__ __forceinline__ unsigned long long kv_globaltimer()
     asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
     return t;
 }
-// bounded wait: gives up after about limit_ns.  A short burst of polls catches HBM-latency waits;
-// after that the thread sleeps between polls, so a CTA that waits on the host link for microseconds
-// at a time does not take issue slots from whatever else runs on its SM.
-__device__ __forceinline__ bool kv_mbar_wait(uint32_t bar, uint32_t parity, unsigned long long limit_ns)
+// bounded wait: `polls` immediate polls, then polls 200 ns apart until about limit_ns have passed.  The
+// short burst catches HBM-latency waits; after that the thread sleeps between polls, so a CTA that waits
+// on the host link for microseconds at a time does not take issue slots from whatever else runs on its
+// SM.  Returns false when the wait ran out (with polls == 0 and limit_ns == 0: without looking at all).
+#define KV_WAIT_POLLS 16u
+#define KV_WAIT_NS 2000000000ull       // 2 s
+__device__ __forceinline__ bool kv_mbar_wait(uint32_t bar, uint32_t parity, unsigned int polls, unsigned long long limit_ns)
 {
 #pragma unroll 1
-    for (int k = 0; k < 16; ++k)
+    for (unsigned int k = 0; k < polls; ++k)
         if (kv_mbar_try_wait(bar, parity)) return true;
+    if (limit_ns == 0) return false;
     const unsigned long long t0 = kv_globaltimer();
     for (;;) {
 #pragma unroll 1
@@ -200,7 +209,6 @@ __global__ void __launch_bounds__(32, 1) kv_copy_bulk(const __grid_constant__ Kv
     long long lo, hi;
     if (!kv_my_range(job, dsel, lo, hi)) return;
     const KvDir &d = job.dir[dsel];
-    constexpr unsigned long long LIMIT_NS = 2000000000ull;   // 2 s per wait
     if (job.t_first) atomicMin(job.t_first, kv_globaltimer());
 
     const uint32_t smem0 = kv_smem_u32(kv_smem);
@@ -231,7 +239,7 @@ __global__ void __launch_bounds__(32, 1) kv_copy_bulk(const __grid_constant__ Kv
         if (j >= 0) {
             const int s = (int)(j % NS);
             const uint32_t parity = (uint32_t)((j / NS) & 1);
-            ok = kv_mbar_wait(bar0 + 8 * s, parity, LIMIT_NS);
+            ok = kv_mbar_wait(bar0 + 8 * s, parity, job.wait_polls, job.wait_ns);
             if (!ok) break;
             ++loads_seen;
             kv_fence_async_smem();
@@ -242,9 +250,10 @@ __global__ void __launch_bounds__(32, 1) kv_copy_bulk(const __grid_constant__ Kv
     }
     if (!ok) {
         atomicOr(job.status, KV_DEV_TIMEOUT);
-        // loads still in flight write into this CTA's shared memory: give each one more bounded wait
+        // loads still in flight write into this CTA's shared memory: give each one more bounded wait (the
+        // fixed bound, whatever the job says) so that none lands after the CTA has gone
         for (long long j = loads_seen; j < loads_issued; ++j)
-            kv_mbar_wait(bar0 + 8 * (int)(j % NS), (uint32_t)((j / NS) & 1), LIMIT_NS);
+            kv_mbar_wait(bar0 + 8 * (int)(j % NS), (uint32_t)((j / NS) & 1), KV_WAIT_POLLS, KV_WAIT_NS);
     }
     kv_bulk_wait_all();
     if (job.t_last) atomicMax(job.t_last, kv_globaltimer());

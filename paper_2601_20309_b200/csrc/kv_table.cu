@@ -125,6 +125,10 @@ struct kv_table {
     std::vector<int64_t> order;     // request ids in arrival order (eager rotation walks it round-robin)
     size_t eager_cursor = 0;
     kv_table_stats_t stats;
+    // test hook (kv_table_fail_pool_call): the pool call that is `fail_after` calls away returns
+    // `fail_code` instead of being made; -1 = not armed
+    int64_t fail_after = -1;
+    int32_t fail_code = KV_OK;
     char err[256];
 };
 
@@ -223,9 +227,32 @@ int32_t take_any_gpu(kv_table *t)
 
 inline int64_t gpu_available(const kv_table *t) { return (int64_t)(t->gpu_free.size() + t->gpu_pending.size()); }
 
-int32_t pool_call(kv_table *t, int32_t rc)
+// Is the pool call about to be made the one a test asked to fail?  (Host-side fault injection: the call
+// is then not made at all, so nothing reaches the device.)
+int32_t injected_failure(kv_table *t)
 {
-    if (rc != KV_OK) snprintf(t->err, 256, "pool call failed (%d): %s", rc, t->pool ? kv_last_error(t->pool) : "");
+    if (t->fail_after < 0) return KV_OK;
+    if (t->fail_after-- > 0) return KV_OK;
+    snprintf(t->err, 256, "pool call failed (%d): injected by kv_table_fail_pool_call", t->fail_code);
+    return t->fail_code;
+}
+
+int32_t pool_swap_out(kv_table *t, const std::vector<int32_t> &og, const std::vector<int32_t> &oh)
+{
+    int32_t rc = injected_failure(t);
+    if (rc != KV_OK || !t->pool) return rc;
+    rc = kv_swap_out(t->pool, og.data(), oh.data(), (int64_t)og.size());
+    if (rc != KV_OK) snprintf(t->err, 256, "pool call failed (%d): %s", rc, kv_last_error(t->pool));
+    return rc;
+}
+
+int32_t pool_rotate(kv_table *t, const std::vector<int32_t> &og, const std::vector<int32_t> &oh,
+                    const std::vector<int32_t> &ih, const std::vector<int32_t> &ig)
+{
+    int32_t rc = injected_failure(t);
+    if (rc != KV_OK || !t->pool) return rc;
+    rc = kv_rotate(t->pool, og.data(), oh.data(), (int64_t)og.size(), ih.data(), ig.data(), (int64_t)ig.size());
+    if (rc != KV_OK) snprintf(t->err, 256, "pool call failed (%d): %s", rc, kv_last_error(t->pool));
     return rc;
 }
 
@@ -335,8 +362,18 @@ int32_t kv_eager_rotate(kv_table_t *t, int64_t max_blocks, int64_t *n_issued)
     if (!t || max_blocks < 0) return KV_ERR_INVALID_ARG;
     std::vector<int32_t> og, oh;
     std::vector<std::pair<int64_t, size_t>> picked;    // (request, block index)
+    std::vector<bool> fresh_host;                      // per picked block: its host id was handed out by this call
     const size_t nreq = t->order.size();
     size_t visited = 0;
+    // all or nothing: if the pool refuses the copy, the host ids handed out here go back and the walk stays put
+    auto undo = [&]() {
+        for (size_t k = picked.size(); k-- > 0;)
+            if (k < fresh_host.size() && fresh_host[k]) {
+                TBlock &b = t->reqs[picked[k].first].blocks[picked[k].second];
+                t->host_free.give(b.h);
+                b.h = -1;
+            }
+    };
     try {
         for (; visited < nreq && (int64_t)picked.size() < max_blocks; ++visited) {
             const int64_t id = t->order[(t->eager_cursor + visited) % nreq];
@@ -346,8 +383,13 @@ int32_t kv_eager_rotate(kv_table_t *t, int64_t max_blocks, int64_t *n_issued)
             for (size_t i = 0; i < r.blocks.size() && (int64_t)(picked.size() + idx.size()) < max_blocks; ++i)
                 if (is_full(t, r, i) && !r.blocks[i].host_valid) idx.push_back(i);
             if (idx.empty()) continue;
+            std::vector<bool> had;
+            for (size_t i : idx) had.push_back(r.blocks[i].h >= 0);
             if (!give_host_ids(t, r, idx)) break;      // host pool exhausted: send what was gathered so far
-            for (size_t i : idx) picked.emplace_back(id, i);
+            for (size_t q = 0; q < idx.size(); ++q) {
+                picked.emplace_back(id, idx[q]);
+                fresh_host.push_back(!had[q]);
+            }
         }
         for (auto &pi : picked) {
             TBlock &b = t->reqs[pi.first].blocks[pi.second];
@@ -355,14 +397,18 @@ int32_t kv_eager_rotate(kv_table_t *t, int64_t max_blocks, int64_t *n_issued)
             oh.push_back(b.h);
         }
     } catch (...) {
+        undo();
         return tfail(t, KV_ERR_NOMEM, "out of host memory");
+    }
+    if (!picked.empty()) {
+        int32_t rc = pool_swap_out(t, og, oh);
+        if (rc != KV_OK) {
+            undo();
+            return rc;
+        }
     }
     if (nreq) t->eager_cursor = (t->eager_cursor + visited) % nreq;
     if (picked.empty()) return KV_OK;
-    if (t->pool) {
-        int32_t rc = pool_call(t, kv_swap_out(t->pool, og.data(), oh.data(), (int64_t)og.size()));
-        if (rc != KV_OK) return rc;
-    }
     for (auto &pi : picked) t->reqs[pi.first].blocks[pi.second].host_valid = true;
     t->stats.eager_blocks += (int64_t)picked.size();
     t->stats.eager_calls++;
@@ -397,6 +443,32 @@ int32_t kv_req_rotate(kv_table_t *t, const int64_t *preempt, int64_t n_preempt, 
 
     std::vector<int32_t> og, oh, ih, ig;
     const TPending seq_before = now(t);             // transfers issued so far may still touch what is released now
+    // All or nothing: steps 1 to 3 work on the table itself (the resuming requests take the very blocks the
+    // preempted ones release), so what they touch is saved first and put back if the pool refuses the rotation.
+    struct Saved {
+        std::vector<int32_t> gpu_free;
+        std::deque<TPending> gpu_pending;
+        ExtentAllocator host_free;
+        std::vector<std::pair<int64_t, std::vector<TBlock>>> blocks;
+        int64_t discarded;
+    } saved;
+    try {
+        saved.gpu_free = t->gpu_free;
+        saved.gpu_pending = t->gpu_pending;
+        saved.host_free = t->host_free;
+        saved.discarded = t->stats.discarded_blocks;
+        for (int64_t k = 0; k < n_preempt; ++k) saved.blocks.emplace_back(preempt[k], t->reqs[preempt[k]].blocks);
+        for (int64_t k = 0; k < n_resume; ++k) saved.blocks.emplace_back(resume[k], t->reqs[resume[k]].blocks);
+    } catch (...) {
+        return tfail(t, KV_ERR_NOMEM, "out of host memory");
+    }
+    auto restore = [&]() {
+        t->gpu_free.swap(saved.gpu_free);
+        t->gpu_pending.swap(saved.gpu_pending);
+        t->host_free = saved.host_free;
+        t->stats.discarded_blocks = saved.discarded;
+        for (auto &sb : saved.blocks) t->reqs[sb.first].blocks.swap(sb.second);
+    };
     try {
         // ---- 1. device blocks that have a valid host copy are released at once, nothing is copied
         for (int64_t k = 0; k < n_preempt; ++k)
@@ -419,19 +491,26 @@ int32_t kv_req_rotate(kv_table_t *t, const int64_t *preempt, int64_t n_preempt, 
             std::vector<size_t> idx;
             for (size_t i = 0; i < r.blocks.size(); ++i)
                 if (!r.blocks[i].host_valid) idx.push_back(i);
-            if (!give_host_ids(t, r, idx)) return tfail(t, KV_ERR_NOMEM, "host pool exhausted");   // excluded by the check above
+            if (!give_host_ids(t, r, idx)) {          // excluded by the check above
+                restore();
+                return tfail(t, KV_ERR_NOMEM, "host pool exhausted");
+            }
             for (size_t i : idx) {
                 og.push_back(r.blocks[i].g);
                 oh.push_back(r.blocks[i].h);
             }
         }
     } catch (...) {
+        restore();
         return tfail(t, KV_ERR_NOMEM, "out of host memory");
     }
     // ---- 4. one rotation: its swap-in destinations are never its swap-out sources (those are still held)
-    if (t->pool && (!og.empty() || !ig.empty())) {
-        int32_t rc = pool_call(t, kv_rotate(t->pool, og.data(), oh.data(), (int64_t)og.size(), ih.data(), ig.data(), (int64_t)ig.size()));
-        if (rc != KV_OK) return rc;
+    if (!og.empty() || !ig.empty()) {
+        int32_t rc = pool_rotate(t, og, oh, ih, ig);
+        if (rc != KV_OK) {
+            restore();
+            return rc;
+        }
     }
     // ---- 5. the sent blocks' device ids are released; this call's swap-out is the one that reads them
     const TPending seq_after = now(t);
@@ -507,6 +586,14 @@ int32_t kv_req_blocks(kv_table_t *t, int64_t req, int32_t *gpu_ids, int32_t *hos
         if (host_ids) host_ids[i] = r->blocks[i].h;
         if (host_valid) host_valid[i] = r->blocks[i].host_valid ? 1 : 0;
     }
+    return KV_OK;
+}
+
+int32_t kv_table_fail_pool_call(kv_table_t *t, int64_t after_calls, int32_t code)
+{
+    if (!t || code >= 0) return KV_ERR_INVALID_ARG;
+    t->fail_after = after_calls < 0 ? -1 : after_calls;
+    t->fail_code = code;
     return KV_OK;
 }
 

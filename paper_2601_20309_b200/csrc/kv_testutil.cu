@@ -9,14 +9,37 @@
 // kvt_checksum_blocks  position-weighted 64-bit sum of the logical content of listed blocks:
 //                      sum over words w at logical index q of w*(2q+1), modulo 2^64.
 //
-// Both take an address rule  address(block, plane) = base + block*blk_stride + plane*plane_stride
+// kvt_wait_runs_out    runs the rotation kernels' bounded barrier wait (kv_mbar_wait of kv_kernels.cuh) on
+//                      a barrier that expects bytes nobody sends, with a short limit: the wait must
+//                      give up after about that long and the kernel must return normally.  This is how
+//                      the give-up branch of the wait is executed without any fault or hang.
+//
+// The first two take an address rule  address(block, plane) = base + block*blk_stride + plane*plane_stride
 // so that they work on the layer-first device pool, the block-first host pool and the
 // layer-first host pool alike.  `base` must be reachable from the device (device memory or
 // mapped pinned host memory).
 #include <cuda_runtime.h>
 #include <stdint.h>
 
+#include "kv_kernels.cuh"
+
 namespace {
+
+// out[0] = 1 if the wait returned "ran out" (else 0), out[1] = nanoseconds the wait took
+__global__ void wait_runs_out_kernel(unsigned long long limit_ns, unsigned long long *out)
+{
+    __shared__ __align__(8) unsigned long long bar;
+    if (threadIdx.x != 0) return;
+    const uint32_t b = kv_smem_u32(&bar);
+    kv_mbar_init(b, 1);
+    kv_fence_mbar_init();
+    kv_mbar_expect_tx(b, 16);                       // the one arrival, and 16 bytes that no copy will ever deliver
+    const unsigned long long t0 = kv_globaltimer();
+    const bool done = kv_mbar_wait(b, 0, KV_WAIT_POLLS, limit_ns);
+    out[1] = kv_globaltimer() - t0;
+    out[0] = done ? 0ull : 1ull;
+    asm volatile("mbarrier.inval.shared::cta.b64 [%0];" ::"r"(b) : "memory");
+}
 
 __device__ __forceinline__ unsigned long long mix64(unsigned long long key)
 {
@@ -113,6 +136,17 @@ int kvt_checksum_blocks(const void *base, long long blk_stride, long long plane_
         checksum_kernel<<<(int)cnt, 256>>>((const unsigned char *)base, blk_stride, plane_stride, words_per_plane,
                                           groups, ids ? ids + lo : nullptr, first_id + lo, out + lo);
     }
+    cudaError_t e = cudaGetLastError();
+    if (e == cudaSuccess) e = cudaDeviceSynchronize();
+    return e == cudaSuccess ? 0 : -(int)e - 1000;
+}
+
+// out: DEVICE pointer to 2 uint64 (see wait_runs_out_kernel).  limit_ns is clamped to 100 ms.  Synchronous.
+int kvt_wait_runs_out(unsigned long long limit_ns, unsigned long long *out)
+{
+    if (!out) return -1;
+    if (limit_ns > 100000000ull) limit_ns = 100000000ull;
+    wait_runs_out_kernel<<<1, 32>>>(limit_ns, out);
     cudaError_t e = cudaGetLastError();
     if (e == cudaSuccess) e = cudaDeviceSynchronize();
     return e == cudaSuccess ? 0 : -(int)e - 1000;

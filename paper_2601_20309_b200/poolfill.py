@@ -25,6 +25,8 @@ def lib() -> C.CDLL:
         L.kvt_fill_blocks.argtypes = [vp, ll, ll, ll, C.c_int, vp, ll, ll, C.c_ulonglong, C.c_ulonglong, vp]
         L.kvt_checksum_blocks.restype = C.c_int
         L.kvt_checksum_blocks.argtypes = [vp, ll, ll, ll, C.c_int, vp, ll, ll, vp]
+        L.kvt_wait_runs_out.restype = C.c_int
+        L.kvt_wait_runs_out.argtypes = [C.c_ulonglong, vp]
         _lib = L
     return _lib
 
@@ -90,3 +92,14 @@ def checksum_words(words: np.ndarray) -> np.uint64:
     w = words.reshape(-1).astype(np.uint64)
     with np.errstate(over="ignore"):
         return (w * (np.uint64(2) * np.arange(len(w), dtype=np.uint64) + np.uint64(1))).sum(dtype=np.uint64)
+
+
+def wait_runs_out(limit_ns: int, device="cuda:0"):
+    """Run the kernels' bounded barrier wait on a barrier nothing completes.  Returns (gave_up, waited_ns)."""
+    import torch
+    out = torch.zeros(2, dtype=torch.int64, device=device)
+    rc = lib().kvt_wait_runs_out(limit_ns, out.data_ptr())
+    if rc != 0:
+        raise RuntimeError(f"kvt_wait_runs_out failed: {rc}")
+    r = out.cpu().numpy()
+    return bool(r[0]), int(r[1])

@@ -509,3 +509,53 @@ def test_caller_streams_and_link_probe():
         B.kv_probe_link_ex(0, copy_bytes=3 << 20, total_bytes=32 << 20, span_bytes=64 << 20, rows=2, host_pitch=1 << 20)
     with pytest.raises(B.KVError):
         B.kv_probe_link_ex(0, copy_bytes=1 << 20, total_bytes=1 << 10, span_bytes=64 << 20)
+
+
+@pytest.mark.parametrize("path", ["zerocopy", "staged"])
+def test_device_leg_is_ordered_against_the_other_direction(path):
+    """kv_gather_blocks / kv_scatter_blocks queued right behind (or in front of) a swap of the other
+    direction that touches the same device blocks, with no kv_sync in between: 200 blocks of 2 MiB, so
+    the first call is still running when the second is issued.  A contiguous device buffer is a
+    block-first pool of its own, so the oracle models a gather as a swap-out into it and a scatter as a
+    swap-in from it."""
+    import torch
+    from oracle.kv_oracle import ByteOracle
+    shape = W.SHAPE_8B
+    n, nbg, nbh = 200, 420, 440
+    p = _pair(shape, nbg, nbh, seed=11, path=PATHS[path])
+    try:
+        rng = np.random.default_rng(4)
+        buf_model = ByteOracle(shape.num_layers, shape.block_size, shape.kv_heads, shape.head_dim, nbg, n, alloc=False)
+        buf_model.G = p.oracle.G                                  # the same device pool
+        buf_model.Hs = rng.integers(0, 256, n * shape.block_bytes, dtype=np.uint8)
+        buf = torch.from_numpy(buf_model.Hs.copy()).to("cuda:0")
+        slots = np.arange(n, dtype=np.int32)
+
+        def check(what):
+            p.assert_equal(what)
+            assert np.array_equal(buf.cpu().numpy(), buf_model.Hs), what + ": the device buffer differs"
+
+        ids = rng.choice(nbg, n, replace=False).astype(np.int32)
+        h1 = rng.choice(nbh, n, replace=False).astype(np.int32)
+        # scatter writes the blocks, the swap-out right behind it must send what the scatter wrote
+        assert buf_model.swap_in(slots, ids) == 0 and p.pool.kv_scatter_blocks(buf.data_ptr(), ids) == 0
+        assert p.oracle.swap_out(ids, h1) == 0 and p.pool.kv_swap_out(ids, h1) == 0
+        check("scatter then swap-out")
+        # swap-in writes the blocks, the gather right behind it must read what came in
+        h2 = rng.choice(nbh, n, replace=False).astype(np.int32)
+        ids2 = rng.choice(nbg, n, replace=False).astype(np.int32)
+        assert p.oracle.swap_in(h2, ids2) == 0 and p.pool.kv_swap_in(h2, ids2) == 0
+        assert buf_model.swap_out(ids2, slots) == 0 and p.pool.kv_gather_blocks(ids2, buf.data_ptr()) == 0
+        check("swap-in then gather")
+        # gather reads the blocks, the swap-in right behind it must not overwrite them too early
+        h3 = rng.choice(nbh, n, replace=False).astype(np.int32)
+        assert buf_model.swap_out(ids, slots) == 0 and p.pool.kv_gather_blocks(ids, buf.data_ptr()) == 0
+        assert p.oracle.swap_in(h3, ids) == 0 and p.pool.kv_swap_in(h3, ids) == 0
+        check("gather then swap-in")
+        # swap-out reads the blocks, the scatter right behind it must wait for it
+        h4 = rng.choice(nbh, n, replace=False).astype(np.int32)
+        assert p.oracle.swap_out(ids2, h4) == 0 and p.pool.kv_swap_out(ids2, h4) == 0
+        assert buf_model.swap_in(slots, ids2) == 0 and p.pool.kv_scatter_blocks(buf.data_ptr(), ids2) == 0
+        check("swap-out then scatter")
+    finally:
+        p.close()
