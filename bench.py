@@ -35,6 +35,7 @@ sys.path.insert(0, ROOT)
 from paper_2601_20309_b200 import metrics as M          # noqa: E402
 from paper_2601_20309_b200 import workload as W         # noqa: E402
 
+CPU_SAMPLE_BLOCKS = 768      # blocks per direction of the rotation that the CPU oracle is timed on, in both arms
 METRIC = "full-duplex KV swap GB/s (out+in)"
 UNIT = "GB/s"
 WORKLOAD = ("config2 llama-3-8b-shaped KV (32 layers, 8 kv heads, head_dim 128, block 16, bf16): "
@@ -188,7 +189,7 @@ def run_reference(args, rank: int) -> None:
         return
     w = W.config2_8b()
     threads = os.cpu_count() or 1
-    nbytes, times, sample = time_oracle(w.shape, w.steps[0], 512, threads, reps=args.steps, warmup=args.warmup)
+    nbytes, times, sample = time_oracle(w.shape, w.steps[0], CPU_SAMPLE_BLOCKS, threads, reps=args.steps, warmup=args.warmup)
     ms = float(np.mean(times)) * 1e3
     val = M.gbs(nbytes, ms)
     line = {"impl": "reference", "metric": METRIC, "value": val, "unit": UNIT, "n_gpus": args.gpus,
@@ -208,6 +209,8 @@ def run_ours(args, rank: int, local_rank: int, world: int) -> None:
 
     if not torch.cuda.is_available():
         raise SystemExit("bench.py needs a CUDA device: the rotation path has no CPU fallback")
+    if local_rank >= torch.cuda.device_count():
+        raise SystemExit(f"bench.py: rank {rank} wants cuda:{local_rank} but the node has {torch.cuda.device_count()} GPUs")
     torch.cuda.set_device(local_rank)
     dev = f"cuda:{local_rank}"
     dist = None
@@ -369,18 +372,38 @@ def run_ours(args, rank: int, local_rank: int, world: int) -> None:
             for k, (a, b) in w.extra[key].items():
                 t = timed((lambda a=a, b=b: pool.kv_swap_out(a, b)) if which == "out" else (lambda a=a, b=b: pool.kv_swap_in(a, b)))
                 singles[f"{which}_{k}"] = {"blocks": len(a), "gbs": M.gbs(len(a) * shape.block_bytes, t), "ms": t}
-        # ---- per-request rotate latency: one request out + one in per call, call entry to completion
-        lat_us, lat_blocks = [], []
-        for r in w.extra["pairs"] * 2:
+        # ---- per-request rotate latency: one request out + one in per call, call entry to completion, host
+        #      clock around the C-ABI calls; all 64 requests (32 pairs), one warm-up pass, then 5 timed passes
+        pair_raw = []
+        for r in w.extra["pairs"]:
             a = tuple(np.ascontiguousarray(x, np.int32) for x in (r.out_gpu, r.out_host, r.in_host, r.in_gpu))
-            raw = (ptr(a[0]), ptr(a[1]), len(a[0]), ptr(a[2]), ptr(a[3]), len(a[3]))
+            pair_raw.append((a, (ptr(a[0]), ptr(a[1]), len(a[0]), ptr(a[2]), ptr(a[3]), len(a[3]))))
+        lat_us, lat_blocks, lat_paths = [], [], {}
+        for rep in range(6):
+            if rep == 1:
+                pool.kv_pool_set_call_timing(False)     # timed by the host clock here: no per-call start events
+            for a, raw in pair_raw:
+                t1 = time.perf_counter()
+                pool.kv_rotate_raw(*raw)
+                pool.kv_sync()
+                dt = (time.perf_counter() - t1) * 1e6
+                if rep:
+                    lat_us.append(dt)
+                    lat_blocks.append(len(a[0]) + len(a[3]))
+                else:
+                    nm = B.PATH_NAMES[pool.kv_get_stats()["last_path_out"]]
+                    lat_paths[nm] = lat_paths.get(nm, 0) + 1
+        # ... and the fixed cost alone: one block each way
+        one = tuple(np.ascontiguousarray(x[:1], np.int32) for x in (og, oh, ih, ig))
+        one_raw = (ptr(one[0]), ptr(one[1]), 1, ptr(one[2]), ptr(one[3]), 1)
+        one_us = []
+        for rep in range(50):
             t1 = time.perf_counter()
-            pool.kv_rotate_raw(*raw)
+            pool.kv_rotate_raw(*one_raw)
             pool.kv_sync()
-            lat_us.append((time.perf_counter() - t1) * 1e6)
-            lat_blocks.append(len(a[0]) + len(a[3]))
-        lat_us = lat_us[len(lat_us) // 2:]       # second pass (first pass warms the path)
-        lat_blocks = lat_blocks[len(lat_blocks) // 2:]
+            if rep >= 10:
+                one_us.append((time.perf_counter() - t1) * 1e6)
+        pool.kv_pool_set_call_timing(True)
         # ---- device-side gather / scatter on their own (HBM <-> contiguous HBM), whole list in one launch
         stage = torch.empty(len(og) * shape.block_bytes, dtype=torch.uint8, device=dev)
         leg = {}
@@ -394,8 +417,89 @@ def run_ours(args, rank: int, local_rank: int, world: int) -> None:
             leg[name] = float(np.mean(ts[3:]))
         leg_bytes = 2.0 * len(og) * shape.block_bytes          # read + write
         del stage
+        p_bi_now = max(probe["bi_sum_gbs"], probe2["bi_sum_gbs"])
+
+        # ---- config 4, the cell of the paper's bandwidth table (section 5.3.3): block 16, 8 GiB (32768 tokens
+        #      of the paper's 256 KB per token) each way, tables random and contiguous; each direction alone
+        #      ("u", end-to-end = the sum) and both at once ("b", end-to-end = the slower one)
+        def table1_cell(contiguous: bool) -> dict:
+            n = int(min(4096, (nb_gpu - 16) // 2, (nb_host - 16) // 2))
+            w4 = W.config4_sweep_case(16, contiguous, n * shape.block_bytes, nb_gpu=nb_gpu, nb_host=nb_host)
+            r4 = w4.steps[0]
+            nb4 = r4.n_out * shape.block_bytes
+            t_o = timed(lambda: pool.kv_swap_out(r4.out_gpu, r4.out_host))
+            t_i = timed(lambda: pool.kv_swap_in(r4.in_host, r4.in_gpu))
+            best = None
+            for _ in range(3):
+                pool.kv_rotate(r4.out_gpu, r4.out_host, r4.in_host, r4.in_gpu)
+                pool.kv_sync()
+                s4 = pool.kv_get_stats()
+                if best is None or s4["last_union_ms"] < best["last_union_ms"]:
+                    best = s4
+            return {"blocks_each_way": int(r4.n_out), "bytes_each_way": nb4,
+                    "d2h_u_gbs": M.gbs(nb4, t_o), "h2d_u_gbs": M.gbs(nb4, t_i), "e2e_ms_serial_u": t_o + t_i,
+                    "d2h_b_gbs": M.gbs(nb4, best["last_out_ms"]), "h2d_b_gbs": M.gbs(nb4, best["last_in_ms"]),
+                    "e2e_ms_concurrent_b": best["last_union_ms"], "both_gbs": M.gbs(2 * nb4, best["last_union_ms"]),
+                    "frac_of_probe": M.gbs(2 * nb4, best["last_union_ms"]) / p_bi_now,
+                    "path": B.PATH_NAMES[best["last_path_out"]]}
+        table1 = {"random_tables": table1_cell(False), "contiguous_tables": table1_cell(True),
+                  "paper_gh200_context": "DuplexKV 180.99 / 179.37 GB/s (b), 46.80 ms; naive 10.75 / 9.86 GB/s (u), 1556.15 ms (Table 1)"}
+
+        # ---- config 5: the serving replay at 8 requests/s under the paper's per-iteration budget of 2400
+        #      blocks; the first 200 steps that move anything, each against the 70 ms of a model step
+        try:
+            w5 = W.config5_replay(rate=8.0, nb_host=min(nb_host, 52888))
+            if w5.nb_gpu > nb_gpu:
+                raise MemoryError("device pool smaller than the replay's")
+            moving = [r5 for r5 in W.budgeted_steps(w5.steps, 2400) if r5.n_out + r5.n_in][:200]
+            ms5, blocks5 = [], []
+            for r5 in moving:
+                pool.kv_rotate(r5.out_gpu, r5.out_host, r5.in_host, r5.in_gpu)
+                pool.kv_sync()
+                ms5.append(pool.kv_get_stats()["last_union_ms"])
+                blocks5.append(r5.n_out + r5.n_in)
+            cfg5 = {"steps_timed": len(ms5), "b_xfer_blocks": 2400, "ms_median": float(np.median(ms5)),
+                    "ms_worst": float(np.max(ms5)), "blocks_median": float(np.median(blocks5)),
+                    "blocks_worst_step": int(blocks5[int(np.argmax(ms5))]),
+                    "gbs_overall": M.gbs(float(np.sum(blocks5)) * shape.block_bytes, float(np.sum(ms5))),
+                    "steps_over_70ms_model_step": int(np.sum(np.array(ms5) > 70.0)),
+                    "model_step_ms_paper": 69.82}
+        except MemoryError as e:
+            cfg5 = {"skipped": f"pools too small on this box: {e}"}
+
+        # ---- config 3: 70B shape (5 MiB blocks, 160 planes), fragmented pool, 8 requests each way per step; a
+        #      second pool over the same device and host memory (already page-locked: no second pinning)
+        cfg3 = None
+        try:
+            s3 = W.SHAPE_70B
+            nb_gpu3 = (nb_gpu * shape.block_bytes) // s3.block_bytes
+            nb_host3 = host_bytes // s3.block_bytes
+            n3 = 12
+            w3 = W.config3_70b(nb_gpu=nb_gpu3, nb_host=nb_host3, n_steps=3 + n3)
+            pool3 = B.KVPool(s3.num_layers, s3.block_size, s3.kv_heads, s3.head_dim, nb_gpu3, nb_host3,
+                             device_pool.data_ptr(), host_base=host_base, device_id=local_rank, path=args.path,
+                             flags=args.flags, staging_bytes=args.staging_mib << 20)
+            ms3, by3 = [], []
+            for k3, r3 in enumerate(w3.steps):
+                pool3.kv_rotate(r3.out_gpu, r3.out_host, r3.in_host, r3.in_gpu)
+                pool3.kv_sync()
+                if k3 >= 3:
+                    ms3.append(pool3.kv_get_stats()["last_union_ms"])
+                    by3.append((r3.n_out + r3.n_in) * s3.block_bytes)
+            st3 = pool3.kv_get_stats()
+            g3 = [M.gbs(b, t) for b, t in zip(by3, ms3)]
+            cfg3 = {"steps_timed": len(ms3), "gpu_pool_blocks": int(nb_gpu3), "host_pool_blocks": int(nb_host3),
+                    "block_bytes": s3.block_bytes, "bytes_per_step_median": float(np.median(by3)),
+                    "ms_per_step_median": float(np.median(ms3)), "gbs_median": float(np.median(g3)),
+                    "gbs_min": float(np.min(g3)), "gbs_max": float(np.max(g3)),
+                    "frac_of_probe": float(np.median(g3)) / p_bi_now, "path": B.PATH_NAMES[st3["last_path_out"]]}
+            pool3.destroy()
+        except (MemoryError, B.KVError) as e:
+            cfg3 = {"skipped": f"not run on this box: {e}"}
+
         extra = {"paths": paths, "singles": singles, "lat_us": lat_us, "lat_blocks": lat_blocks, "leg": leg,
-                 "leg_bytes": leg_bytes, "probe2": probe2, "contiguous_host": contiguous_host, "table": tb}
+                 "leg_bytes": leg_bytes, "probe2": probe2, "contiguous_host": contiguous_host, "table": tb,
+                 "lat_paths": lat_paths, "one_us": one_us, "table1": table1, "cfg5": cfg5, "cfg3": cfg3}
 
     pool.destroy()
     del device_pool
@@ -404,7 +508,7 @@ def run_ours(args, rank: int, local_rank: int, world: int) -> None:
     if rank == 0:
         # ---- CPU oracle on the host cores, bounded sample of the same rotation
         threads = os.cpu_count() or 1
-        nb_s, t_mt, sample = time_oracle(shape, rot, 768, threads, reps=20, warmup=2)
+        nb_s, t_mt, sample = time_oracle(shape, rot, CPU_SAMPLE_BLOCKS, threads, reps=20, warmup=2)
         _, t_1, _ = time_oracle(shape, rot, 256, 1, reps=5)
         cpu_val = M.gbs(nb_s, float(np.mean(t_mt)) * 1e3)
         cpu_1 = M.gbs(2 * 256 * shape.block_bytes, float(np.mean(t_1)) * 1e3)
@@ -435,7 +539,10 @@ def run_ours(args, rank: int, local_rank: int, world: int) -> None:
                         "algorithmic_bytes_per_launch": 2.0 * k_bytes / k_n,
                         "peak_source": f"MEASURED_PEAKS.json hbm_gbs ({peaks['source']}; burst copy figure)",
                         "frac_of_nominal_8TBs": k_ach / 8000.0,
-                        "how": "CUDA events around every pack / unpack launch on the stream it runs on, inside the timed steps",
+                        "how": "CUDA events around every pack / unpack launch on the stream it runs on, inside the timed steps. "
+                               "The step itself is bound by the host link, not by this kernel (its launches take "
+                               f"{100.0 * k_ms / dev_total_ms:.1f} % of the step): the step's own fraction is "
+                               f"roofline_link.frac = {value / world / p_bi:.3f} of the probed both-directions rate",
                         # the same launches timed from inside the kernel (first CTA start to last CTA end): the
                         # events also see the wait for the launch, which is long while the link is busy
                         "exec_only": {"achieved": M.gbs(2.0 * k_bytes, k_exec_ms), "avg_launch_us": k_exec_ms / k_n * 1e3,
@@ -480,8 +587,16 @@ def run_ours(args, rank: int, local_rank: int, world: int) -> None:
             "block_table": extra["table"],
             "single_swaps": extra["singles"],
             "request_rotate_us": {"p50": M.percentile(extra["lat_us"], 0.5), "p99": M.percentile(extra["lat_us"], 0.99),
-                                  "n": len(extra["lat_us"]),
-                                  "median_blocks_per_call": float(np.median(extra["lat_blocks"]))},
+                                  "n": len(extra["lat_us"]), "requests": 2 * len(w.extra["pairs"]), "passes": 5,
+                                  "median_blocks_per_call": float(np.median(extra["lat_blocks"])),
+                                  "paths_taken": extra["lat_paths"],
+                                  "how": "host clock from kv_rotate entry to kv_sync return, one request out + one in per call"},
+            "one_block_rotate_us": {"p50": M.percentile(extra["one_us"], 0.5), "p99": M.percentile(extra["one_us"], 0.99),
+                                    "n": len(extra["one_us"]),
+                                    "link_time_us": shape.block_bytes / (p_d2h * 1e9) * 1e6},
+            "config3": extra["cfg3"],
+            "config4_table1": extra["table1"],
+            "config5": extra["cfg5"],
             "cpu_baseline": {"value": cpu_val, "unit": UNIT, "cores": threads, "kind": "oracle", "sample": sample,
                              "single_thread_value": cpu_1},
         }
@@ -508,6 +623,10 @@ def main() -> None:
     args = ap.parse_args()
     if args.warmup < 3 and args.impl == "ours":
         args.warmup = 3
+    if args.gpus > 1 and "WORLD_SIZE" not in os.environ and args.impl == "ours":
+        # not started by a launcher: start the N replicas here, one process per GPU
+        from paper_2601_20309_b200 import replicas as R
+        sys.exit(R.main_spawn(args.gpus))
     rank = int(os.environ.get("RANK", "0"))
     local_rank = int(os.environ.get("LOCAL_RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))

@@ -58,8 +58,10 @@ extern "C" {
 #define KV_DEV_BLOCK_FIRST    1     /* [block][layer][K|V]...: the paper's redesigned storage order      */
 
 /* transfer paths (how the host link is driven) */
-#define KV_PATH_AUTO          0     /* per call: STAGED when the copy-engine transfers the call needs would
-                                       average 3 MiB or more, else ZEROCOPY (see kv_path_for)            */
+#define KV_PATH_AUTO          0     /* per call.  Calls bound by fixed costs: CE2D when the call moves 8 MiB
+                                       or less per direction, ZEROCOPY up to 24 MiB.  Larger calls: STAGED
+                                       when the copy-engine transfers the call needs would average 3 MiB
+                                       or more, else ZEROCOPY (see kv_path_for)                          */
 #define KV_PATH_ZEROCOPY      1     /* SM kernels read/write mapped pinned host memory directly          */
 #define KV_PATH_STAGED        2     /* pack kernel -> contiguous HBM staging -> copy engine (and reverse)*/
 #define KV_PATH_CE2D          3     /* one strided 2-D copy-engine transfer per block, no kernel         */
@@ -71,7 +73,9 @@ extern "C" {
 #define KV_FLAG_LDST_KERNEL     2   /* ZEROCOPY/STAGED kernels use plain 16-byte loads/stores instead of
                                        bulk asynchronous copies through shared memory                    */
 #define KV_FLAG_FUSED_ROTATE    4   /* ZEROCOPY kv_rotate with disjoint lists: one launch, CTAs split
-                                       between the directions, on the out stream                         */
+                                       between the directions, on the out stream.  Without the flag this
+                                       is done only for short lists (64 blocks or fewer each way) on an
+                                       idle pool, where it saves a launch; longer ones use two streams   */
 #define KV_FLAG_TIME_KERNELS    8   /* bracket every HBM-to-HBM gather / scatter kernel (STAGED pack / unpack,
                                        kv_gather_blocks, kv_scatter_blocks) with events on its own stream;
                                        kv_sync adds their durations to the timed_* statistics            */
@@ -85,7 +89,11 @@ typedef struct {
                                borrowed (typically a torch tensor's storage)                              */
     void   *host_base;      /* HOST pointer or NULL.  NULL: the library allocates num_host_blocks*BLK
                                bytes of mapped pinned memory and owns it.  Non-NULL: caller memory of that
-                               size, 4096-byte aligned; the library page-locks it for the pool's lifetime */
+                               size, 4096-byte aligned; the library page-locks it for the pool's lifetime.
+                               Memory that is page-locked already (all of it: by cudaHostAlloc or
+                               cudaHostRegister, or because it is the host memory of another pool) is
+                               used as it is, which spares the seconds page-locking takes per 10 GB
+                               when several pools of different shapes share one host buffer in turn     */
     int32_t host_layout;    /* KV_HOST_BLOCK_FIRST or KV_HOST_LAYER_FIRST                                 */
     int32_t device_id;
     void   *stream_out;     /* cudaStream_t or NULL (library creates a non-blocking stream)               */
@@ -113,8 +121,10 @@ typedef struct {
     int64_t calls_out, calls_in;       /* data-moving calls per direction                                 */
     int64_t kernel_launches;           /* kernels this library launched                                   */
     int64_t ce_copies;                 /* copy-engine transfers this library issued                       */
-    double  last_out_ms, last_in_ms;   /* device time of the latest completed call per direction,
-                                          from events on the launching streams; valid after kv_sync       */
+    double  last_out_ms, last_in_ms;   /* device time of the latest completed call per direction, from
+                                          events on the launching streams.  Computed by kv_get_stats for
+                                          the latest call a kv_sync has waited for: read the statistics
+                                          after that kv_sync and before the next data-moving call          */
     double  last_union_ms;             /* first start to last end of the latest call (both directions
                                           for kv_rotate)                                                  */
     int32_t last_path_out, last_path_in;
@@ -202,6 +212,11 @@ int32_t kv_plan_staged(int64_t blk_bytes, int64_t half_blocks, int32_t direction
  * re-applies the rule of kv_path_for).  Pool contents are unaffected. */
 int32_t kv_pool_set_path(kv_pool_t *pool, int32_t path_out, int32_t path_in);
 
+/* Waits for outstanding work, then switches the per-call timing on (default) or off.  Off: calls record no
+ * start events and the last_* statistics stay as they are, which takes a few microseconds off every call;
+ * for callers that rotate single requests and time them with their own clock.  (Tuning of this library.) */
+int32_t kv_pool_set_call_timing(kv_pool_t *pool, int32_t on);
+
 /*
  * Bound of the waits inside the copy kernels (each wait of a kernel's main loop for a load it has
  * issued): `polls` immediate polls, then polls 200 ns apart for at most `ns` nanoseconds (default 16 and
@@ -215,7 +230,8 @@ int32_t kv_pool_set_path(kv_pool_t *pool, int32_t path_out, int32_t path_in);
 int32_t kv_pool_set_wait_limit(kv_pool_t *pool, uint32_t polls, uint64_t ns);
 
 /* Wait for both directions.  Returns KV_OK, or the first sticky asynchronous error
- * (KV_ERR_CUDA, KV_ERR_TIMEOUT).  Fills the last_* timing fields of the statistics. */
+ * (KV_ERR_CUDA, KV_ERR_TIMEOUT).  The last_* timing fields describe the call it waited for once
+ * kv_get_stats is called. */
 int32_t kv_sync(kv_pool_t *pool);
 
 /*

@@ -105,7 +105,7 @@ EXPORTS = ["kv_pool_create", "kv_pool_destroy", "kv_pool_set_path", "kv_swap_out
            "kv_table_create", "kv_table_create_dry", "kv_table_destroy", "kv_table_last_error", "kv_req_add",
            "kv_req_append", "kv_eager_rotate", "kv_req_rotate", "kv_req_preempt", "kv_req_resume", "kv_req_finish",
            "kv_req_info", "kv_req_blocks", "kv_table_get_stats", "kv_table_fail_pool_call",
-           "kv_pool_set_wait_limit"]
+           "kv_pool_set_wait_limit", "kv_pool_set_call_timing"]
 
 _lib = None
 
@@ -184,6 +184,8 @@ def lib() -> C.CDLL:
     L.kv_req_blocks.argtypes = [vp, i64, i32p, i32p, C.POINTER(C.c_uint8), i64]
     L.kv_table_get_stats.restype = C.c_int32
     L.kv_table_get_stats.argtypes = [vp, C.POINTER(kv_table_stats_t)]
+    L.kv_pool_set_call_timing.restype = C.c_int32
+    L.kv_pool_set_call_timing.argtypes = [vp, C.c_int32]
     L.kv_pool_set_wait_limit.restype = C.c_int32
     L.kv_pool_set_wait_limit.argtypes = [vp, C.c_uint32, C.c_uint64]
     L.kv_table_fail_pool_call.restype = C.c_int32
@@ -348,6 +350,9 @@ class KVPool:
 
     def kv_pool_set_path(self, path_out: int, path_in: int, check: bool = True) -> int:
         return self._ret(lib().kv_pool_set_path(self._h, path_out, path_in), check)
+
+    def kv_pool_set_call_timing(self, on: bool, check: bool = True) -> int:
+        return self._ret(lib().kv_pool_set_call_timing(self._h, int(on)), check)
 
     def kv_pool_set_wait_limit(self, polls: int, ns: int, check: bool = True) -> int:
         return self._ret(lib().kv_pool_set_wait_limit(self._h, polls, ns), check)

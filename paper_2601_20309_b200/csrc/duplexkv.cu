@@ -21,7 +21,15 @@ namespace {
 constexpr int KV_SLOTS = 8;            // descriptor / event ring depth per direction
 constexpr int KV_MAX_CE_STREAMS = 4;
 constexpr int64_t KV_AUTO_MIN_TRANSFER = 3ll << 20;   // AUTO: staged when its transfers average 3 MiB or more
-constexpr int64_t KV_MERGE_MIN_MEAN_RUN = 8;          // STAGED: merge runs of host ids when they average 8 blocks or more
+// AUTO, calls bound by fixed costs rather than by the link (measured on 2 MiB blocks, scattered ids, call to
+// completion): up to 8 MiB per direction one copy-engine transfer per block is quickest (73 / 117 / 232 us for
+// 1 / 2 / 4 blocks each way against 92 / 148 / 251 us for the zero-copy kernels, whose duplex rate is lower);
+// up to 24 MiB the zero-copy kernels are (462 us at 8 blocks against 470 and 496); from 32 MiB on the staged
+// pipeline is ahead and the transfer-size rule below decides.
+constexpr int64_t KV_AUTO_TINY_BYTES = 8ll << 20;
+constexpr int64_t KV_AUTO_SMALL_BYTES = 24ll << 20;
+constexpr int64_t KV_MERGE_MIN_MEAN_RUN = 8;
+constexpr int64_t KV_PLAN_CHUNKS = 4;                 // STAGED: a call that fits one staging half is still cut into about this many chunks          // STAGED: merge runs of host ids when they average 8 blocks or more
 constexpr int BULK_STAGE = 16384;      // bytes per shared-memory stage of the bulk kernel
 constexpr int BULK_NS = 8;             // stages
 constexpr int BULK_AHEAD = 5;          // loads in flight ahead of the stores
@@ -105,9 +113,11 @@ struct kv_pool {
     uint32_t epoch = 0;
     std::vector<uint64_t> g_read_by_out, g_written_by_in, h_written_by_out, h_read_by_in;
     kv_stats_t stats;
-    bool union_valid = false;
+    bool union_valid = false;          // the latest call's events have not been turned into statistics yet
+    bool union_synced = false;         // ... and kv_sync has seen that call complete
     int union_slot[2] = {-1, -1};      // slots of the latest call (per direction; -1 = not part of it)
     int32_t sticky = KV_OK;
+    bool call_timing = true;           // record per-call start events and keep the last_* statistics (kv_pool_set_call_timing)
     unsigned int wait_polls = KV_WAIT_POLLS;            // bound of the kernels' main-loop waits (kv_pool_set_wait_limit)
     unsigned long long wait_ns = KV_WAIT_NS;
     char err[256];
@@ -380,6 +390,21 @@ struct PlanParams {
     bool layer_first;           // host pool layout
 };
 
+// Where the sorted list is cut into chunks: chunk number k holds `first` blocks, then twice as much each
+// time, up to `chunk`; the boundaries depend on n alone and no transfer crosses one.  With `even`, chunks
+// hold an even number of blocks (two-block transfers are never split into singles).
+std::vector<int64_t> chunk_bounds(int64_t n, int64_t first, int64_t chunk, bool even)
+{
+    std::vector<int64_t> bounds{0};
+    while (bounds.back() < n) {
+        const size_t k = bounds.size() - 1;
+        int64_t take = k < 40 ? std::min(chunk, first << k) : chunk;
+        if (even && take > 1) take &= ~(int64_t)1;
+        bounds.push_back(std::min(n, bounds.back() + take));
+    }
+    return bounds;
+}
+
 // Pure planning (no pool, no CUDA): order, transfers and chunks for n pairs of direction d (0 out, 1 in)
 // whose host block ids are host_ids.  May throw std::bad_alloc.
 // mode: -1 = decide from this list's runs, 0 = merge runs, 1 = uniform two-block transfers;
@@ -399,12 +424,13 @@ void plan_transfers(const PlanParams &pp, int d, const int32_t *host_ids, int64_
         // own packing, transfers and unpacking overlap instead of following one another.  The first chunk
         // of a swap-out is half as long as the rest: its first transfer starts sooner.
         const int64_t min_chunk = std::max<int64_t>(1, (8ll << 20) / pp.blk);
-        const int64_t chunk = std::min(pp.half_blocks, std::max(min_chunk, (n + 3) / 4));
+        const int64_t chunk = std::min(pp.half_blocks, std::max(min_chunk, (n + KV_PLAN_CHUNKS - 1) / KV_PLAN_CHUNKS));
         const int64_t first = (d == 0 && n > chunk) ? std::max<int64_t>(1, chunk / 2) : chunk;
         if (pp.layer_first) {
             // one strided transfer per block: `planes` rows of SEG bytes, a whole host plane apart
-            for (int64_t lo = 0, hi = 0; lo < n; lo = hi) {
-                hi = std::min(n, lo + (lo == 0 ? first : chunk));
+            const std::vector<int64_t> bounds = chunk_bounds(n, first, chunk, false);
+            for (size_t q = 0; q + 1 < bounds.size(); ++q) {
+                const int64_t lo = bounds[q], hi = bounds[q + 1];
                 CeChunk ch{lo, hi, (int32_t)ops.size(), 0};
                 for (int64_t k = lo; k < hi; ++k)
                     ops.push_back(CeOp{(int64_t)host_ids[order[(size_t)k]] * pp.seg, (k - lo) * pp.blk, pp.seg,
@@ -414,7 +440,7 @@ void plan_transfers(const PlanParams &pp, int d, const int32_t *host_ids, int64_
             }
             return;
         }
-        // ---- 1. transfers over the sorted list, none longer than a chunk.
+        // Transfers over the sorted list, chunk by chunk.
         // Measured with both directions busy: transfers that all carry the same number of bytes keep the
         // two copy engines in step and share the link evenly (2 x 2 MiB everywhere: 93.9 GB/s), while a
         // mix of sizes loses 8 % (85.6 GB/s for mostly pairs with a few singles and triples), whatever
@@ -428,45 +454,33 @@ void plan_transfers(const PlanParams &pp, int d, const int32_t *host_ids, int64_
         const bool uniform = mode < 0 ? n < KV_MERGE_MIN_MEAN_RUN * nruns : mode == 1;
         if (nruns_out) *nruns_out = nruns;
         if (uniform_out) *uniform_out = uniform;
-        auto run_len = [&](int64_t q) {
-            int64_t r = 1;
-            if (uniform) return r;
-            while (q + r < n && r < chunk && hid(q + r) == hid(q) + r) ++r;
-            return r;
-        };
-        for (int64_t k = 0; k < n;) {
-            const int64_t r = run_len(k);
-            CeOp op{hid(k) * pp.blk, 0, r * pp.blk, r * pp.blk, 1, k, (int32_t)r};
-            int64_t nxt = k + r;
-            // further runs of the same length at a constant spacing join as extra rows (uniform mode: one)
-            while (nxt < n && op.nblk + r <= chunk && run_len(nxt) == r && !(uniform && op.rows >= 2)) {
-                const int64_t pitch = (hid(nxt) - hid(nxt - r)) * pp.blk;
-                if (pitch < op.width || pitch > pp.max_pitch || (op.rows > 1 && pitch != op.host_pitch)) break;
-                op.host_pitch = pitch;
-                op.rows++;
-                op.nblk += (int32_t)r;
-                nxt += r;
+        const std::vector<int64_t> bounds = chunk_bounds(n, first, chunk, uniform);
+        for (size_t q = 0; q + 1 < bounds.size(); ++q) {
+            const int64_t lo = bounds[q], hi = bounds[q + 1];
+            auto run_len = [&](int64_t k) {
+                int64_t r = 1;
+                if (uniform) return r;
+                while (k + r < hi && hid(k + r) == hid(k) + r) ++r;
+                return r;
+            };
+            CeChunk ch{lo, hi, (int32_t)ops.size(), 0};
+            for (int64_t k = lo; k < hi;) {
+                const int64_t r = run_len(k);
+                // the staging slot of sorted position k is (k - lo) * BLK into the chunk's half
+                CeOp op{hid(k) * pp.blk, (k - lo) * pp.blk, r * pp.blk, r * pp.blk, 1, k, (int32_t)r};
+                int64_t nxt = k + r;
+                // further runs of the same length at a constant spacing join as extra rows (uniform mode: one)
+                while (nxt < hi && run_len(nxt) == r && nxt + r <= hi && !(uniform && op.rows >= 2)) {
+                    const int64_t pitch = (hid(nxt) - hid(nxt - r)) * pp.blk;
+                    if (pitch < op.width || pitch > pp.max_pitch || (op.rows > 1 && pitch != op.host_pitch)) break;
+                    op.host_pitch = pitch;
+                    op.rows++;
+                    op.nblk += (int32_t)r;
+                    nxt += r;
+                }
+                ops.push_back(op);
+                k = nxt;
             }
-            ops.push_back(op);
-            k = nxt;
-        }
-        // ---- 2. staging slots follow the sorted order; chunks are cut when a staging half is full
-        int64_t filled = 0;
-        CeChunk ch{0, 0, 0, 0};
-        for (size_t a = 0; a < ops.size(); ++a) {
-            CeOp &op = ops[a];
-            const int64_t cap = chunks.empty() ? first : chunk;
-            if (filled > ch.lo && filled - ch.lo + op.nblk > cap) {
-                ch.hi = filled;
-                ch.op_hi = (int32_t)a;
-                chunks.push_back(ch);
-                ch = CeChunk{filled, filled, (int32_t)a, 0};
-            }
-            op.stage_off = (filled - ch.lo) * pp.blk;
-            filled += op.nblk;
-        }
-        if (filled > ch.lo) {
-            ch.hi = filled;
             ch.op_hi = (int32_t)ops.size();
             chunks.push_back(ch);
         }
@@ -512,7 +526,7 @@ int32_t begin_dir(kv_pool *p, DirCall &c, cudaEvent_t wait_for)
     DirState &s = p->dir[c.d];
     const uint64_t seq = s.issued + 1;
     c.slot = (int)(seq % KV_SLOTS);
-    if (seq > KV_SLOTS) KV_CUDA(p, cudaEventSynchronize(s.ev_end[c.slot]));   // slot's previous user
+    if (seq > KV_SLOTS && s.done + KV_SLOTS < seq) KV_CUDA(p, cudaEventSynchronize(s.ev_end[c.slot]));   // slot's previous user
     c.pairs_host = s.ring_host + (size_t)c.slot * 2 * p->cap;
     c.pairs_dev = s.ring_dev + (size_t)c.slot * 2 * p->cap;
     c.aux_host = c.pairs_host + p->cap;
@@ -523,14 +537,16 @@ int32_t begin_dir(kv_pool *p, DirCall &c, cudaEvent_t wait_for)
             const int32_t g = c.gpu_ids[s.order[(size_t)k]];
             c.aux_host[k] = (c.d == 0) ? make_int2(g, (int)k) : make_int2((int)k, g);
         }
-    } else if (c.path == KV_PATH_ZEROCOPY) {
+    } else if (c.path == KV_PATH_ZEROCOPY && c.n > KV_INLINE_PAIRS) {
         for (int64_t i = 0; i < c.n; ++i)
             c.pairs_host[i] = (c.d == 0) ? make_int2(c.gpu_ids[i], c.host_ids[i]) : make_int2(c.host_ids[i], c.gpu_ids[i]);
     }
     if (wait_for) KV_CUDA(p, cudaStreamWaitEvent(s.stream, wait_for, 0));
-    KV_CUDA(p, cudaEventRecord(s.ev_start[c.slot], s.stream));
+    if (p->call_timing) KV_CUDA(p, cudaEventRecord(s.ev_start[c.slot], s.stream));
     if (c.path == KV_PATH_ZEROCOPY) {
-        KV_CUDA(p, cudaMemcpyAsync(c.pairs_dev, c.pairs_host, (size_t)c.n * sizeof(int2), cudaMemcpyHostToDevice, s.stream));
+        // a short list travels in the launch parameters instead (zerocopy_dir)
+        if (c.n > KV_INLINE_PAIRS)
+            KV_CUDA(p, cudaMemcpyAsync(c.pairs_dev, c.pairs_host, (size_t)c.n * sizeof(int2), cudaMemcpyHostToDevice, s.stream));
     } else if (c.path == KV_PATH_STAGED) {
         KV_CUDA(p, cudaMemcpyAsync(c.aux_dev, c.aux_host, (size_t)c.n * sizeof(int2), cudaMemcpyHostToDevice, s.stream));
         // the kernel stream starts after everything issued so far on this direction
@@ -572,15 +588,21 @@ int32_t end_dir(kv_pool *p, DirCall &c)
     return KV_OK;
 }
 
-KvDir zerocopy_dir(kv_pool *p, const DirCall &c)
+// direction `k` of `job` := the zero-copy description of call c
+void zerocopy_dir(kv_pool *p, const DirCall &c, KvJob &job, int k)
 {
-    KvDir d;
+    KvDir &d = job.dir[k];
     d.src = (c.d == 0) ? device_side(p) : host_side(p);
     d.dst = (c.d == 0) ? host_side(p) : device_side(p);
-    d.pairs = c.pairs_dev;
     d.n = (int)c.n;
     d.ctas = 0;
-    return d;
+    if (c.n <= KV_INLINE_PAIRS) {
+        d.pairs = nullptr;
+        for (int64_t i = 0; i < c.n; ++i)
+            job.inl[k][i] = (c.d == 0) ? make_int2(c.gpu_ids[i], c.host_ids[i]) : make_int2(c.host_ids[i], c.gpu_ids[i]);
+    } else {
+        d.pairs = c.pairs_dev;
+    }
 }
 
 // host address of the start of host block h (block-first) or of its first plane (layer-first)
@@ -704,8 +726,8 @@ int32_t issue_calls(kv_pool *p, DirCall *calls, int ncalls, bool fused)
     if (fused && ncalls == 2 && calls[0].path == KV_PATH_ZEROCOPY && calls[1].path == KV_PATH_ZEROCOPY) {
         KvJob job;
         fill_geometry(p, job, true);
-        job.dir[0] = zerocopy_dir(p, calls[0]);
-        job.dir[1] = zerocopy_dir(p, calls[1]);
+        zerocopy_dir(p, calls[0], job, 0);
+        zerocopy_dir(p, calls[1], job, 1);
         job.dir[0].ctas = clamp_ctas(job, job.dir[0], p->dir[0].ctas);
         job.dir[1].ctas = clamp_ctas(job, job.dir[1], p->dir[1].ctas);
         KV_CUDA(p, launch_job(p, job, p->dir[0].stream, true));
@@ -716,7 +738,7 @@ int32_t issue_calls(kv_pool *p, DirCall *calls, int ncalls, bool fused)
         if (c.path != KV_PATH_ZEROCOPY) continue;
         KvJob job;
         fill_geometry(p, job, true);
-        job.dir[0] = zerocopy_dir(p, c);
+        zerocopy_dir(p, c, job, 0);
         job.dir[1] = KvDir{};
         job.dir[0].ctas = clamp_ctas(job, job.dir[0], p->dir[c.d].ctas);
         KV_CUDA(p, launch_job(p, job, p->dir[c.d].stream, true));
@@ -734,7 +756,9 @@ int32_t issue_calls(kv_pool *p, DirCall *calls, int ncalls, bool fused)
     return KV_OK;
 }
 
-int32_t run_calls(kv_pool *p, DirCall *calls, int ncalls, const bool *wait_other, bool fused)
+// may_fuse: the caller (kv_rotate with lists that do not overlap and wait for nothing) allows both
+// directions to share one launch; whether they do is decided here, once the paths are known.
+int32_t run_calls(kv_pool *p, DirCall *calls, int ncalls, const bool *wait_other, bool may_fuse)
 {
     p->union_slot[0] = p->union_slot[1] = -1;
     // The event each call has to wait for is the end of the other direction's latest EARLIER call.  It is
@@ -747,23 +771,46 @@ int32_t run_calls(kv_pool *p, DirCall *calls, int ncalls, const bool *wait_other
             const DirState &o = p->dir[1 - calls[k].d];
             wait_ev[k] = o.ev_end[o.issued % KV_SLOTS];
         }
-    // KV_PATH_AUTO is settled per call: plan the staged transfers first (cheap: a sort of the ids), and
-    // take the staged path when its transfers would carry KV_AUTO_MIN_TRANSFER bytes or more on average,
-    // the zero-copy kernels otherwise.  Both directions of a rotate take the same path (a kernel on one
-    // direction starves the copy engine on the other).
+    // KV_PATH_AUTO is settled per call.  A call that moves little is bound by its fixed costs, not by the
+    // link: up to KV_AUTO_TINY_BYTES per direction it goes as one copy-engine transfer per block, up to
+    // KV_AUTO_SMALL_BYTES to the zero-copy kernels (one launch, no staging pipeline).  Otherwise the staged
+    // transfers are planned first (cheap: a sort of the ids) and the staged path is taken when its transfers
+    // would carry KV_AUTO_MIN_TRANSFER bytes or more on average, the zero-copy kernels when not.  Both
+    // directions of a rotate take the same path (a kernel on one direction starves the copy engine on the
+    // other).
     {
-        int64_t bytes = 0, ops = 0;
+        int64_t largest = 0;
         for (int k = 0; k < ncalls; ++k) {
             calls[k].path = p->dir[calls[k].d].path;
-            if (calls[k].path != KV_PATH_AUTO) continue;
-            int32_t rc = plan_staged(p, calls[k]);
-            if (rc != KV_OK) return rc;
-            bytes += calls[k].n * p->blk;
-            ops += (int64_t)p->dir[calls[k].d].ops.size();
+            if (calls[k].path == KV_PATH_AUTO) largest = std::max(largest, calls[k].n * p->blk);
         }
-        const int chosen = (ops > 0 && bytes >= ops * KV_AUTO_MIN_TRANSFER) ? KV_PATH_STAGED : KV_PATH_ZEROCOPY;
+        int chosen;
+        if (largest <= KV_AUTO_TINY_BYTES) {
+            chosen = KV_PATH_CE2D;
+        } else if (largest <= KV_AUTO_SMALL_BYTES) {
+            chosen = KV_PATH_ZEROCOPY;
+        } else {
+            int64_t bytes = 0, ops = 0;
+            for (int k = 0; k < ncalls; ++k) {
+                if (calls[k].path != KV_PATH_AUTO) continue;
+                int32_t rc = plan_staged(p, calls[k]);
+                if (rc != KV_OK) return rc;
+                bytes += calls[k].n * p->blk;
+                ops += (int64_t)p->dir[calls[k].d].ops.size();
+            }
+            chosen = (ops > 0 && bytes >= ops * KV_AUTO_MIN_TRANSFER) ? KV_PATH_STAGED : KV_PATH_ZEROCOPY;
+        }
         for (int k = 0; k < ncalls; ++k)
             if (calls[k].path == KV_PATH_AUTO) calls[k].path = chosen;
+    }
+    // One launch for both directions of a zero-copy rotate: always when the pool asks for it
+    // (KV_FLAG_FUSED_ROTATE), and by itself when both lists are short and nothing else is in flight on
+    // the pool -- then the call is all fixed cost, and one launch on one stream is the least of it.
+    bool fused = false;
+    if (may_fuse && ncalls == 2 && calls[0].path == KV_PATH_ZEROCOPY && calls[1].path == KV_PATH_ZEROCOPY) {
+        const bool small = calls[0].n <= KV_INLINE_PAIRS && calls[1].n <= KV_INLINE_PAIRS;
+        const bool idle = p->dir[0].done >= p->dir[0].issued && p->dir[1].done >= p->dir[1].issued;
+        fused = (p->cfg.flags & KV_FLAG_FUSED_ROTATE) || (small && idle);
     }
     // Both directions of a staged rotate use the same kind of transfers: two-block transfers one way and
     // long merged ones the other way fall out of step (74 GB/s measured against 88 to 95 when alike).
@@ -821,6 +868,34 @@ int32_t run_calls(kv_pool *p, DirCall *calls, int ncalls, const bool *wait_other
     for (int k = 0; k < ncalls; ++k) p->union_slot[calls[k].d] = calls[k].slot;
     p->union_valid = true;
     return KV_OK;
+}
+
+// Turn the start / end events of the latest call into the last_* statistics.  Done when the statistics
+// are read, not in kv_sync: four event queries are a measurable part of a small rotation's latency.
+void harvest_call_timing(kv_pool *p)
+{
+    if (!p->union_valid || !p->union_synced) return;
+    float t_out = 0.f, t_in = 0.f, off = 0.f;
+    const int so = p->union_slot[0], si = p->union_slot[1];
+    if (so >= 0) (void)cudaEventElapsedTime(&t_out, p->dir[0].ev_start[so], p->dir[0].ev_end[so]);
+    if (si >= 0) (void)cudaEventElapsedTime(&t_in, p->dir[1].ev_start[si], p->dir[1].ev_end[si]);
+    if (so >= 0) p->stats.last_out_ms = t_out;
+    if (si >= 0) p->stats.last_in_ms = t_in;
+    if (so >= 0 && si >= 0) {
+        // position of the in-window relative to the out-window; either may start first
+        float a = 0.f, b = 0.f;
+        const bool fwd = cudaEventElapsedTime(&a, p->dir[0].ev_start[so], p->dir[1].ev_start[si]) == cudaSuccess;
+        const bool bwd = cudaEventElapsedTime(&b, p->dir[1].ev_start[si], p->dir[0].ev_start[so]) == cudaSuccess;
+        off = (fwd && a > 0.f) ? a : ((bwd && b > 0.f) ? -b : 0.f);
+        const float lo = std::min(0.f, off), hi = std::max(t_out, off + t_in);
+        p->stats.last_union_ms = hi - lo;
+        p->stats.last_in_offset_ms = off;
+    } else {
+        p->stats.last_union_ms = so >= 0 ? t_out : t_in;
+        p->stats.last_in_offset_ms = 0.0;
+    }
+    (void)cudaGetLastError();
+    p->union_valid = p->union_synced = false;
 }
 
 }  // namespace
@@ -914,13 +989,18 @@ int32_t kv_pool_create(const kv_pool_config_t *cfg, kv_pool_t **out)
     if (cfg->host_base) {
         p->host = (uint8_t *)cfg->host_base;
         cudaError_t e = cudaHostRegister(p->host, host_bytes, cudaHostRegisterMapped | cudaHostRegisterPortable);
-        if (e != cudaSuccess) {
+        if (e == cudaErrorHostMemoryAlreadyRegistered) {
+            // page-locked already (by the caller, or it is another pool's host memory): used as it is and
+            // left page-locked at destroy
+            (void)cudaGetLastError();
+        } else if (e != cudaSuccess) {
             (void)cudaGetLastError();
             int32_t rc = fail(nullptr, KV_ERR_NOMEM, "cudaHostRegister of host_base failed");
             kv_pool_destroy(p);
             return rc;
+        } else {
+            p->registered_host = true;
         }
-        p->registered_host = true;
     } else {
         cudaError_t e = cudaHostAlloc((void **)&p->host, host_bytes, cudaHostAllocMapped | cudaHostAllocPortable);
         if (e != cudaSuccess) {
@@ -1102,9 +1182,7 @@ int32_t kv_rotate(kv_pool_t *p, const int32_t *out_gpu, const int32_t *out_host,
         calls[1].n = n_in;
         const bool wait[2] = {conflicts_with_other(p, 0, out_gpu, out_host, n_out),
                               conflicts_with_other(p, 1, in_gpu, in_host, n_in)};
-        const bool fused = (p->cfg.flags & KV_FLAG_FUSED_ROTATE) && p->dir[0].path == KV_PATH_ZEROCOPY &&
-                           p->dir[1].path == KV_PATH_ZEROCOPY && !wait[0] && !wait[1];
-        return run_calls(p, calls, 2, wait, fused);
+        return run_calls(p, calls, 2, wait, !wait[0] && !wait[1]);
     }
     // overlap allowed: the conflict-free swap-ins run beside the swap-out, the others after it
     std::vector<int32_t> free_h, free_g, conf_h, conf_g;
@@ -1197,6 +1275,16 @@ int32_t kv_pool_set_path(kv_pool_t *p, int32_t path_out, int32_t path_in)
     return KV_OK;
 }
 
+int32_t kv_pool_set_call_timing(kv_pool_t *p, int32_t on)
+{
+    if (!p) return KV_ERR_INVALID_ARG;
+    int32_t rc = kv_sync(p);
+    if (rc != KV_OK) return rc;
+    p->call_timing = on != 0;
+    p->union_valid = p->union_synced = false;
+    return KV_OK;
+}
+
 int32_t kv_pool_set_wait_limit(kv_pool_t *p, uint32_t polls, uint64_t ns)
 {
     if (!p) return KV_ERR_INVALID_ARG;
@@ -1214,29 +1302,7 @@ int32_t kv_sync(kv_pool_t *p)
         if (e != cudaSuccess) return fail_cuda(p, e, "cudaStreamSynchronize");
         p->dir[d].done = p->dir[d].issued;
     }
-    if (p->union_valid) {
-        float t_out = 0.f, t_in = 0.f, off = 0.f;
-        const int so = p->union_slot[0], si = p->union_slot[1];
-        if (so >= 0) (void)cudaEventElapsedTime(&t_out, p->dir[0].ev_start[so], p->dir[0].ev_end[so]);
-        if (si >= 0) (void)cudaEventElapsedTime(&t_in, p->dir[1].ev_start[si], p->dir[1].ev_end[si]);
-        if (so >= 0) p->stats.last_out_ms = t_out;
-        if (si >= 0) p->stats.last_in_ms = t_in;
-        if (so >= 0 && si >= 0) {
-            // position of the in-window relative to the out-window; either may start first
-            float a = 0.f, b = 0.f;
-            const bool fwd = cudaEventElapsedTime(&a, p->dir[0].ev_start[so], p->dir[1].ev_start[si]) == cudaSuccess;
-            const bool bwd = cudaEventElapsedTime(&b, p->dir[1].ev_start[si], p->dir[0].ev_start[so]) == cudaSuccess;
-            off = (fwd && a > 0.f) ? a : ((bwd && b > 0.f) ? -b : 0.f);
-            const float lo = std::min(0.f, off), hi = std::max(t_out, off + t_in);
-            p->stats.last_union_ms = hi - lo;
-            p->stats.last_in_offset_ms = off;
-        } else {
-            p->stats.last_union_ms = so >= 0 ? t_out : t_in;
-            p->stats.last_in_offset_ms = 0.0;
-        }
-        (void)cudaGetLastError();
-        p->union_valid = false;
-    }
+    if (p->union_valid) p->union_synced = true;     // kv_get_stats turns the events into the last_* fields
     for (int d = 0; d < 2; ++d) {
         DirState &s = p->dir[d];
         if (s.kev_used > 0 && s.ktime_dev) {
@@ -1294,7 +1360,7 @@ static int32_t device_leg(kv_pool_t *p, const int32_t *gpu_ids, int64_t n, const
     }
     const uint64_t seq = s.issued + 1;
     const int slot = (int)(seq % KV_SLOTS);
-    if (seq > KV_SLOTS) KV_CUDA(p, cudaEventSynchronize(s.ev_end[slot]));
+    if (seq > KV_SLOTS && s.done + KV_SLOTS < seq) KV_CUDA(p, cudaEventSynchronize(s.ev_end[slot]));
     int2 *ph = s.ring_host + (size_t)slot * 2 * p->cap;
     int2 *pd = s.ring_dev + (size_t)slot * 2 * p->cap;
     for (int64_t i = 0; i < n; ++i) ph[i] = (d == 0) ? make_int2(gpu_ids[i], (int)i) : make_int2((int)i, gpu_ids[i]);
@@ -1318,6 +1384,7 @@ static int32_t device_leg(kv_pool_t *p, const int32_t *gpu_ids, int64_t n, const
     p->union_slot[d] = slot;
     p->union_slot[1 - d] = -1;
     p->union_valid = true;
+    p->union_synced = false;
     return KV_OK;
 }
 
@@ -1378,6 +1445,7 @@ int32_t kv_host_ptr(kv_pool_t *p, void **base, int64_t *bytes)
 int32_t kv_get_stats(kv_pool_t *p, kv_stats_t *st)
 {
     if (!p || !st) return KV_ERR_INVALID_ARG;
+    harvest_call_timing(p);
     p->stats.device_status = *(volatile unsigned int *)p->status_host;
     *st = p->stats;
     return KV_OK;

@@ -36,10 +36,13 @@ struct KvSide {
 
 struct KvDir {
     KvSide src, dst;
-    const int2 *pairs;   // x = source block id, y = destination block id (device memory)
+    const int2 *pairs;   // x = source block id, y = destination block id (device memory);
+                         // nullptr = the list is short and travels with the launch (KvJob::inl)
     int n;               // pairs
     int ctas;            // CTAs assigned to this direction (0 = direction absent)
 };
+
+#define KV_INLINE_PAIRS 64   // longest pair list carried in the kernel parameters (1 KiB for both directions)
 
 struct KvJob {
     KvDir dir[2];
@@ -55,7 +58,16 @@ struct KvJob {
     // optional: device words that receive the earliest start and the latest end of the launch's CTAs
     // (%globaltimer, ns); nullptr = not wanted.  The host presets them to ~0 and 0.
     unsigned long long *t_first, *t_last;
+    // pair lists of at most KV_INLINE_PAIRS entries ride in the launch parameters: a small rotation then
+    // needs no separate copy of its ids, and the kernel no read from memory to find its first block
+    int2 inl[2][KV_INLINE_PAIRS];
 };
+
+__device__ __forceinline__ int2 kv_pair(const KvJob &job, int dsel, int i)
+{
+    const int2 *pairs = job.dir[dsel].pairs;
+    return pairs ? pairs[i] : job.inl[dsel][i];
+}
 
 // ------------------------------------------------------------------------------------------------
 // work-item cursor: (pair i, plane p, chunk c), advanced one item at a time
@@ -63,23 +75,25 @@ struct KvCursor {
     int i, p, c;
     int2 pr;
 
-    __device__ __forceinline__ void seek(const KvJob &job, const KvDir &d, long long item)
+    __device__ __forceinline__ void seek(const KvJob &job, int dsel, long long item)
     {
+        const KvDir &d = job.dir[dsel];
         const long long per = (long long)job.planes * job.cps;
         i = (int)(item / per);
         const int r = (int)(item - (long long)i * per);
         p = r / job.cps;
         c = r - p * job.cps;
-        pr = (i < d.n) ? d.pairs[i] : make_int2(0, 0);
+        pr = (i < d.n) ? kv_pair(job, dsel, i) : make_int2(0, 0);
     }
-    __device__ __forceinline__ void step(const KvJob &job, const KvDir &d)
+    __device__ __forceinline__ void step(const KvJob &job, int dsel)
     {
+        const KvDir &d = job.dir[dsel];
         if (++c == job.cps) {
             c = 0;
             if (++p == job.planes) {
                 p = 0;
                 ++i;
-                if (i < d.n) pr = d.pairs[i];
+                if (i < d.n) pr = kv_pair(job, dsel, i);
             }
         }
     }
@@ -219,7 +233,7 @@ __global__ void __launch_bounds__(32, 1) kv_copy_bulk(const __grid_constant__ Kv
     kv_fence_async_smem();
 
     KvCursor ld, st;
-    ld.seek(job, d, lo);
+    ld.seek(job, dsel, lo);
     st = ld;
     const long long n_items = hi - lo;
     long long loads_issued = 0, loads_seen = 0;
@@ -232,7 +246,7 @@ __global__ void __launch_bounds__(32, 1) kv_copy_bulk(const __grid_constant__ Kv
             const uint32_t nbytes = (uint32_t)ld.bytes(job);
             kv_mbar_expect_tx(bar0 + 8 * s, nbytes);
             kv_bulk_load(smem0 + s * STAGE, ld.src(job, d), nbytes, bar0 + 8 * s);
-            ld.step(job, d);
+            ld.step(job, dsel);
             ++loads_issued;
         }
         const long long j = k - AHEAD;
@@ -245,7 +259,7 @@ __global__ void __launch_bounds__(32, 1) kv_copy_bulk(const __grid_constant__ Kv
             kv_fence_async_smem();
             kv_bulk_store(st.dst(job, d), smem0 + s * STAGE, (uint32_t)st.bytes(job));
             kv_bulk_commit();
-            st.step(job, d);
+            st.step(job, dsel);
         }
     }
     if (!ok) {
@@ -277,12 +291,12 @@ __global__ void __launch_bounds__(THREADS) kv_copy_ldst(const __grid_constant__ 
     int p = r / job.cps;
     int c = r - p * job.cps;
     int win = i;
-    int2 mine = (win + lane < d.n) ? d.pairs[win + lane] : make_int2(0, 0);
+    int2 mine = (win + lane < d.n) ? kv_pair(job, dsel, win + lane) : make_int2(0, 0);
 
     for (long long item = lo; item < hi; ++item) {
         if (i >= win + 32) {
             win = i;
-            mine = (win + lane < d.n) ? d.pairs[win + lane] : make_int2(0, 0);
+            mine = (win + lane < d.n) ? kv_pair(job, dsel, win + lane) : make_int2(0, 0);
         }
         const int sid = __shfl_sync(0xffffffffu, mine.x, i - win);
         const int did = __shfl_sync(0xffffffffu, mine.y, i - win);

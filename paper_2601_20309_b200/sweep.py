@@ -19,8 +19,9 @@
 
     python -m paper_2601_20309_b200.sweep latency [--out FILE]
         Call-to-completion time of small rotations (1 .. 256 blocks each way, 8B shape, scattered ids):
-        host clock around kv_rotate + kv_sync, median of 40, per path.  What a per-request rotate costs
-        when the link is not the limit.
+        host clock around kv_rotate + kv_sync through the C ABI with ready-made id arrays, median of 40,
+        per path, and how much of it the call itself takes before it returns.  What a per-request
+        rotate costs when the link is not the limit, and whether AUTO picks the quickest path.
 
     python -m paper_2601_20309_b200.sweep budget [--b-xfer N] [--out FILE]
         The serving replay (8B shape, 8 requests/s, 2000 steps) re-timed under the paper's per-iteration
@@ -221,31 +222,42 @@ def latency(out) -> None:
     dev = torch.empty(nb * shape.block_bytes, dtype=torch.uint8, device="cuda:0")
     pool = B.KVPool(shape.num_layers, shape.block_size, shape.kv_heads, shape.head_dim, nb, nb, dev.data_ptr())
     rng = np.random.default_rng(3)
+    i32p = B.C.POINTER(B.C.c_int32)
     rows = []
-    for n in (1, 2, 4, 8, 16, 64, 256):
+    for n in (1, 2, 4, 8, 16, 32, 64, 128, 256):
         pg, ph = rng.permutation(nb).astype(np.int32), rng.permutation(nb).astype(np.int32)
-        og, ig, oh, ih = pg[:n], pg[n:2 * n], ph[:n], ph[n:2 * n]
+        og, ig, oh, ih = (np.ascontiguousarray(x) for x in (pg[:n], pg[n:2 * n], ph[:n], ph[n:2 * n]))
+        raw = (og.ctypes.data_as(i32p), oh.ctypes.data_as(i32p), n, ih.ctypes.data_as(i32p), ig.ctypes.data_as(i32p), n)
         rec = {"blocks_each_way": n, "mib_each_way": n * shape.block_bytes / M}
         for name, pid in (("auto", B.KV_PATH_AUTO), ("staged", B.KV_PATH_STAGED), ("zerocopy", B.KV_PATH_ZEROCOPY),
-                          ("ce2d", B.KV_PATH_CE2D)):
+                          ("ce2d", B.KV_PATH_CE2D), ("auto_untimed", B.KV_PATH_AUTO)):
             pool.kv_pool_set_path(pid, pid)
-            ts = []
+            pool.kv_pool_set_call_timing(name != "auto_untimed")       # last column: no per-call start events
+            ts, issue = [], []
             for k in range(45):
                 t0 = time.perf_counter()
-                pool.kv_rotate(og, oh, ih, ig)
+                pool.kv_rotate_raw(*raw)
+                t1 = time.perf_counter()
                 pool.kv_sync()
+                t2 = time.perf_counter()
                 if k >= 5:
-                    ts.append((time.perf_counter() - t0) * 1e6)
+                    ts.append((t2 - t0) * 1e6)
+                    issue.append((t1 - t0) * 1e6)
             rec[name + "_us"] = round(float(np.median(ts)), 1)
+            rec[name + "_issue_us"] = round(float(np.median(issue)), 1)
             if name == "auto":
                 rec["auto_took"] = B.PATH_NAMES[pool.kv_get_stats()["last_path_out"]]
         rec["link_floor_us"] = round(n * shape.block_bytes / 50e9 * 1e6, 1)       # payload at 50 GB/s per direction
+        best = min(rec[k + "_us"] for k in ("staged", "zerocopy", "ce2d"))
+        rec["auto_over_best_pct"] = round(100 * (rec["auto_us"] / best - 1), 1)
         rows.append(rec)
         _emit(rec, out)
     pool.destroy()
-    print("\n| blocks each way | MiB each way | AUTO us (took) | staged us | zero-copy us | 2-D per block us | payload at 50 GB/s per direction, us |\n|---|---|---|---|---|---|---|")
+    print("\n| blocks each way | MiB each way | AUTO us (took; of which issuing) | staged us | zero-copy us | 2-D per block us | "
+          "AUTO over the best fixed path | AUTO, call timing off, us | payload at 50 GB/s per direction, us |\n|---|---|---|---|---|---|---|---|---|")
     for r in rows:
-        print(f"| {r['blocks_each_way']} | {r['mib_each_way']:g} | {r['auto_us']} ({r['auto_took']}) | {r['staged_us']} | {r['zerocopy_us']} | {r['ce2d_us']} | {r['link_floor_us']} |")
+        print(f"| {r['blocks_each_way']} | {r['mib_each_way']:g} | {r['auto_us']} ({r['auto_took']}; {r['auto_issue_us']}) | {r['staged_us']} | "
+              f"{r['zerocopy_us']} | {r['ce2d_us']} | {r['auto_over_best_pct']} % | {r['auto_untimed_us']} | {r['link_floor_us']} |")
 
 
 def budget(out, b_xfer: int) -> None:

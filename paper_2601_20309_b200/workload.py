@@ -385,7 +385,8 @@ def config2_8b(seed: int = MASTER_SEED + 2, nb_gpu: Optional[int] = None, nb_hos
     """8B-shaped KV; 64 requests with lognormal lengths (median 1k tokens, max 8k), half resident
     on each side.  ``steps[0]`` is the paired rotation of 16 requests each way; ``extra`` holds the
     single swap-out / swap-in lists (median-length and longest request) and one-pair-at-a-time
-    rotations of the other requests for per-request latency."""
+    rotations of every request (first the other 32, then the 32 of the paired rotation on their way
+    back) for per-request latency."""
     rng = np.random.default_rng(seed)
     nb_gpu = blocks_for_bytes(shape, 60e9) if nb_gpu is None else nb_gpu
     nb_host = blocks_for_bytes(shape, 120e9) if nb_host is None else nb_host
@@ -416,6 +417,9 @@ def config2_8b(seed: int = MASTER_SEED + 2, nb_gpu: Optional[int] = None, nb_hos
     extra = {"single_out": single(gpu_rids, "gpu"), "single_in": single(host_rids, "host")}
     rot = tab.rotate(g_rot, h_rot)
     extra["pairs"] = [tab.rotate([a], [b]) for a, b in zip(g_rest, h_rest)]
+    # ... and the requests of the paired rotation change places once more, one pair at a time, so that
+    # all ``n_req`` requests take part in a one-request-each-way rotation (per-request latency sample)
+    extra["pairs"] += [tab.rotate([b], [a]) for a, b in zip(g_rot, h_rot)]
     extra["tokens"] = toks
     return Workload("8b", shape, nb_gpu, nb_host, seed, tab, [rot], extra)
 
@@ -594,3 +598,150 @@ def budgeted_steps(steps: Sequence[Rotation], b_xfer: int) -> List[Rotation]:
     while queue:
         emit()
     return out
+
+
+# --------------------------------------------------------------------------- lists made by the paper's scheduler
+#
+# The paper drives its rotation engine with a scheduler (section 4.2): every request has a Virtual Lag
+# Time (VLT), and each engine iteration the Largest-VLT-First policy (Algorithm 1) picks the requests to
+# bring onto the GPU and the running requests to preempt for them.  Here the policy is only a maker of
+# rotation lists: a seeded toy loop over synthetic arrivals, no SLO study.
+
+@dataclass(frozen=True)
+class LVFParams:
+    """Scheduler settings of the paper's evaluation (section 5.2): alpha = 3, beta_B = 0, beta_F = 0.5,
+    B_xfer = 2400 blocks, first-token SLO 5 s, between-token SLO 100 ms.  ``slo_first_s`` is the S_F and
+    ``slo_between_s`` the S_B of the VLT definition (F: first token, B: between tokens)."""
+    alpha: float = 3.0
+    beta_b: float = 0.0
+    beta_f: float = 0.5
+    slo_first_s: float = 5.0
+    slo_between_s: float = 0.100
+    b_xfer: int = 2400
+
+
+def vlt(state: str, t_now: float, t_ref: float, p: LVFParams = LVFParams()) -> float:
+    """Virtual Lag Time of one request (section 4.2, the piecewise definition).  ``t_ref`` is the time of
+    the last generated token for a rotary request, the arrival time for a waiting one, and the time it
+    entered the running state for a running one."""
+    if state == "rotary":
+        return p.alpha * max(0.0, t_now - t_ref - p.beta_b * p.slo_between_s)
+    if state == "waiting":
+        return max(0.0, t_now - t_ref - p.beta_f * p.slo_first_s)
+    if state == "running":
+        return -(t_now - t_ref)
+    raise ValueError(state)
+
+
+def lvf_select(requests: Sequence[Tuple[int, str, float, int]], b_hbm: int, b_xfer: int) -> Tuple[List[int], List[int]]:
+    """One decision of Largest-VLT-First (Algorithm 1).  ``requests`` holds (id, state, VLT, blocks) with
+    state in {"running", "waiting", "rotary"}; ``b_hbm`` is the number of free device blocks.  Returns
+    (preempted ids, prioritized ids), each in the order the algorithm picks them.
+
+    Steps, as the paper numbers them: (1) if the free blocks hold every waiting and rotary request, nothing
+    is preempted and all of them are prioritized; (2) sort everything by VLT, largest first; (3) from the
+    head, take waiting / rotary requests whose blocks still fit into ``b_hbm + b_xfer``; (4) the blocks
+    needed beyond the free ones are ``B_swap``: from the tail, preempt running requests until that many
+    are freed.  Equal VLTs keep the order of ``requests`` (a stable sort)."""
+    idle = [r for r in requests if r[1] != "running"]
+    if b_hbm >= sum(r[3] for r in idle):
+        return [], [r[0] for r in idle]
+    order = sorted(requests, key=lambda r: -r[2])
+    left = b_hbm + b_xfer
+    prioritized = []
+    for rid, state, v, blk in order:
+        if state != "running" and v >= 0 and blk <= left:
+            prioritized.append(rid)
+            left -= blk
+    swap = b_xfer - left
+    preempted = []
+    for rid, state, v, blk in reversed(order):
+        if state == "running" and v < 0 and swap > 0:
+            preempted.append(rid)
+            swap -= blk
+    return preempted, prioritized
+
+
+def config5_lvf(seed: int = MASTER_SEED + 6, rate: float = 8.0, n_steps: int = 2000, shape: KVShape = SHAPE_8B,
+                duration_s: float = 120.0, step_s: float = 0.070, nb_host: Optional[int] = None, cap: float = 0.40,
+                max_tokens: int = 8192, params: LVFParams = LVFParams()) -> Workload:
+    """The serving replay of ``config5_replay`` (same arrivals, lengths, growth of one token per running
+    request per 70 ms step, device pool at 40 % of the unconstrained demand) with the paper's scheduler
+    choosing who moves: each step computes every request's VLT and runs one Largest-VLT-First decision
+    under the free-block count and ``params.b_xfer``.
+
+    What a decision turns into.  Preempted requests are swapped out in this step.  A prioritized rotary
+    request is swapped in, and a prioritized waiting request is admitted (its prompt blocks allocated, no
+    transfer), only as far as blocks are free *before* this step's swap-out releases any: the lists take
+    swap-in destinations from the free list first, so no rotation ever names a block in both directions
+    (the paper gets the same freedom from eager block rotation; without it the blocks a preemption frees
+    serve the next step).  Requests left over stay in their queue and are decided on again next step.
+    ``extra`` reports how many requests each step preempted / resumed / admitted."""
+    rng = np.random.default_rng(seed)
+    n_arr = max(1, int(rng.poisson(rate * duration_s)))
+    arrive = np.sort(rng.uniform(0.0, duration_s, size=n_arr))
+    prompt = lognormal_tokens(rng, n_arr, 512, 1, max_tokens)
+    output = lognormal_tokens(rng, n_arr, 256, 1, max_tokens)
+    bs = shape.block_size
+    nblk = lambda tokens: -(-int(tokens) // bs)
+    a_step = np.floor(arrive / step_s).astype(np.int64)
+    horizon = int(a_step.max() + output.max() + 2)
+    delta = np.zeros(horizon + 1, np.int64)
+    for s, p_, o in zip(a_step, prompt, output):
+        delta[s] += nblk(p_ + o)
+        delta[min(horizon, s + int(o))] -= nblk(p_ + o)
+    demand = int(np.cumsum(delta).max())
+    nb_gpu = max(int(cap * demand), nblk((prompt + output).max()) + 8)
+    nb_host = max(2 * demand, 64) if nb_host is None else nb_host
+    tab = RequestTable(shape, nb_gpu, nb_host, rng)
+    running: Dict[int, float] = {}         # rid -> time it entered the running state
+    rotary: Dict[int, float] = {}          # rid -> time of its last generated token
+    waiting: List[int] = []                # arrival order
+    remaining: Dict[int, int] = {}
+    steps: List[Rotation] = []
+    log = {"preempted": [], "resumed": [], "admitted": [], "deferred": []}
+    nxt = 0
+    for step in range(n_steps):
+        t_now = step * step_s
+        while nxt < n_arr and a_step[nxt] <= step:
+            waiting.append(nxt)
+            nxt += 1
+        for rid in [r for r in running if remaining[r] <= 0]:
+            del running[rid]
+            tab.finish(rid)
+        grow_need = sum(1 for r in running if tab.requests[r].tokens % bs == 0)
+        b_hbm = max(0, len(tab.gpu_free) - grow_need)
+        reqs = [(r, "running", vlt("running", t_now, t0, params), len(tab.requests[r].blocks)) for r, t0 in running.items()]
+        reqs += [(r, "waiting", vlt("waiting", t_now, float(arrive[r]), params), nblk(prompt[r])) for r in waiting]
+        reqs += [(r, "rotary", vlt("rotary", t_now, t0, params), len(tab.requests[r].blocks)) for r, t0 in rotary.items()]
+        preempt, prio = lvf_select(reqs, b_hbm, params.b_xfer)
+        blk_of = {r[0]: r[3] for r in reqs}
+        free_now = b_hbm
+        ins, admit, deferred = [], [], 0
+        for rid in prio:
+            if blk_of[rid] > free_now:
+                deferred += 1
+                continue
+            free_now -= blk_of[rid]
+            (ins if rid in rotary else admit).append(rid)
+        steps.append(tab.rotate(preempt, ins) if (preempt or ins) else _empty_rotation())
+        for rid in preempt:
+            del running[rid]
+            rotary[rid] = t_now
+        for rid in ins:
+            del rotary[rid]
+            running[rid] = t_now
+        for rid in admit:
+            waiting.remove(rid)
+            tab.add(rid, int(prompt[rid]), "gpu")
+            remaining[rid] = int(output[rid])
+            running[rid] = t_now
+        for k, v in (("preempted", len(preempt)), ("resumed", len(ins)), ("admitted", len(admit)), ("deferred", deferred)):
+            log[k].append(v)
+        for rid in running:
+            if tab.requests[rid].tokens % bs == 0 and len(tab.gpu_free) == 0:
+                continue                       # stalled this step: no block to grow into
+            tab.grow(rid, tab.requests[rid].tokens + 1)
+            remaining[rid] -= 1
+    return Workload(f"lvf_{rate:g}rps", shape, nb_gpu, nb_host, seed, tab, steps,
+                    {"demand_blocks": demand, "arrivals": n_arr, **{k: np.asarray(v) for k, v in log.items()}})

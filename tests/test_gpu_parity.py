@@ -559,3 +559,20 @@ def test_device_leg_is_ordered_against_the_other_direction(path):
         check("swap-out then scatter")
     finally:
         p.close()
+
+
+def test_lists_made_by_the_lvf_scheduler_match_the_oracle():
+    """Rotation lists that the paper's Largest-VLT-First policy produces on synthetic arrivals (a CPU toy
+    that only makes inputs), first 300 steps on a shrunk shape, queued without syncing, AUTO path."""
+    w = W.config5_lvf(rate=3.0, n_steps=300, shape=W.KVShape(2, 16, 2, 64), duration_s=20.0, max_tokens=1024,
+                      params=W.LVFParams(b_xfer=40))
+    assert sum(1 for s in w.steps if s.n_out and s.n_in) > 10
+    p = _pair(w.shape, w.nb_gpu, w.nb_host, seed=w.seed, path=0)
+    try:
+        for k, r in enumerate(w.steps):
+            assert p.rotate_both(r) == 0
+            if k % 100 == 99:
+                p.assert_equal(f"LVF step {k}")
+        p.assert_equal("LVF final")
+    finally:
+        p.close()

@@ -78,7 +78,7 @@ def test_equal_runs_at_a_constant_spacing_share_one_strided_transfer():
     ids = np.concatenate([np.arange(s, s + 16) for s in range(100, 100 + 8 * 40, 40)])            # 8 runs of 16, 40 apart
     ops, _ = check_plan(ids, 512, 0)
     assert any(op["rows"] > 1 and op["blocks_per_row"] == 16 and op["pitch_blocks"] == 40 for op in ops)
-    assert len(ops) <= 4
+    assert len(ops) <= 5                                                     # chunks of 16, 32, 32, 32, 16 blocks
 
 
 def test_repeated_sources_far_apart_ids_and_tiny_lists():

@@ -50,3 +50,28 @@ def test_two_replicas_add_bytes_and_take_the_slowest_time():
 def test_single_process_is_the_identity():
     assert M.reduce_over_ranks(3.5, "max") == 3.5
     assert M.replicas_gbs(2e9, 1000.0) == pytest.approx(2.0)
+
+
+def test_launcher_starts_one_replica_per_rank_and_passes_rank_zero_through():
+    """What ``bench.py --gpus N`` does when no launcher started it: N processes with the rendezvous
+    variables set, rank 0's single JSON line as the only output."""
+    import json
+    import sys
+    from paper_2601_20309_b200 import replicas as R
+    stub = os.path.join(os.path.dirname(os.path.abspath(__file__)), "stub_replica.py")
+    codes, text = R.spawn(2, [sys.executable, stub], timeout_s=240, capture=True)
+    assert codes == [0, 0]
+    lines = [ln for ln in text.splitlines() if ln.strip()]
+    assert len(lines) == 1
+    rec = json.loads(lines[0])
+    assert rec["n_gpus"] == 2
+    assert rec["value"] == pytest.approx((4.0e9 + 6.0e9) / 0.075 / 1e9)     # bytes added, slowest rank's time
+    codes, _ = R.spawn(2, [sys.executable, stub, "--fail-rank", "1"], timeout_s=240, capture=True)
+    assert codes == [0, 3]                                                  # a failing rank is reported
+
+
+def test_rank_environment():
+    from paper_2601_20309_b200 import replicas as R
+    env = R.rank_env(3, 8, 29511, base={"KEEP": "1"})
+    assert env == {"KEEP": "1", "RANK": "3", "LOCAL_RANK": "3", "WORLD_SIZE": "8", "LOCAL_WORLD_SIZE": "8",
+                   "MASTER_ADDR": "127.0.0.1", "MASTER_PORT": "29511"}

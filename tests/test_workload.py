@@ -58,7 +58,11 @@ def test_config2_8b_full_size_lists():
     assert len(r.out_req_offsets) == 17 and len(r.in_req_offsets) == 17
     assert abs(r.n_out - r.n_in) < 0.05 * r.n_out            # a rotation frees about what it brings in
     assert not set(r.in_gpu) & set(r.out_gpu)
-    assert len(w.extra["pairs"]) == 16
+    pairs = w.extra["pairs"]
+    assert len(pairs) == 32                                   # every one of the 64 requests rotates once, pairwise
+    moved = sum(len(p.out_req_offsets) - 1 + len(p.in_req_offsets) - 1 for p in pairs)
+    assert moved == 64 and all(p.n_out and p.n_in and not set(p.in_gpu) & set(p.out_gpu) for p in pairs)
+    assert sum(p.n_out + p.n_in for p in pairs) == sum(-(-int(t) // 16) for t in toks)
     for k in ("median", "longest"):
         src, dst = w.extra["single_out"][k]
         assert len(src) == len(dst) and len(set(dst)) == len(dst)
