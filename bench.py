@@ -254,7 +254,7 @@ def run_ours(args, rank: int, local_rank: int, world: int) -> None:
     pool = B.KVPool(shape.num_layers, shape.block_size, shape.kv_heads, shape.head_dim, nb_gpu, nb_host,
                     device_pool.data_ptr(), device_id=local_rank, path=args.path,
                     flags=args.flags | B.KV_FLAG_TIME_KERNELS, ctas_out=args.ctas, ctas_in=args.ctas,
-                    staging_bytes=args.staging_mib << 20)
+                    staging_bytes=args.staging_mib << 20, link_variant=args.link_variant)
     pin_s = time.perf_counter() - t0
     host_base, host_bytes = pool.kv_host_ptr()
     # seeded content in both pools (GPU twin of the CPU generator; verified against it in the tests);
@@ -419,83 +419,85 @@ def run_ours(args, rank: int, local_rank: int, world: int) -> None:
         del stage
         p_bi_now = max(probe["bi_sum_gbs"], probe2["bi_sum_gbs"])
 
-        # ---- config 4, the cell of the paper's bandwidth table (section 5.3.3): block 16, 8 GiB (32768 tokens
-        #      of the paper's 256 KB per token) each way, tables random and contiguous; each direction alone
-        #      ("u", end-to-end = the sum) and both at once ("b", end-to-end = the slower one)
-        def table1_cell(contiguous: bool) -> dict:
-            n = int(min(4096, (nb_gpu - 16) // 2, (nb_host - 16) // 2))
-            w4 = W.config4_sweep_case(16, contiguous, n * shape.block_bytes, nb_gpu=nb_gpu, nb_host=nb_host)
-            r4 = w4.steps[0]
-            nb4 = r4.n_out * shape.block_bytes
-            t_o = timed(lambda: pool.kv_swap_out(r4.out_gpu, r4.out_host))
-            t_i = timed(lambda: pool.kv_swap_in(r4.in_host, r4.in_gpu))
-            best = None
-            for _ in range(3):
-                pool.kv_rotate(r4.out_gpu, r4.out_host, r4.in_host, r4.in_gpu)
-                pool.kv_sync()
-                s4 = pool.kv_get_stats()
-                if best is None or s4["last_union_ms"] < best["last_union_ms"]:
-                    best = s4
-            return {"blocks_each_way": int(r4.n_out), "bytes_each_way": nb4,
-                    "d2h_u_gbs": M.gbs(nb4, t_o), "h2d_u_gbs": M.gbs(nb4, t_i), "e2e_ms_serial_u": t_o + t_i,
-                    "d2h_b_gbs": M.gbs(nb4, best["last_out_ms"]), "h2d_b_gbs": M.gbs(nb4, best["last_in_ms"]),
-                    "e2e_ms_concurrent_b": best["last_union_ms"], "both_gbs": M.gbs(2 * nb4, best["last_union_ms"]),
-                    "frac_of_probe": M.gbs(2 * nb4, best["last_union_ms"]) / p_bi_now,
-                    "path": B.PATH_NAMES[best["last_path_out"]]}
-        table1 = {"random_tables": table1_cell(False), "contiguous_tables": table1_cell(True),
-                  "paper_gh200_context": "DuplexKV 180.99 / 179.37 GB/s (b), 46.80 ms; naive 10.75 / 9.86 GB/s (u), 1556.15 ms (Table 1)"}
+        table1, cfg5, cfg3 = None, None, None
+        if not args.quick:
+            # ---- config 4, the cell of the paper's bandwidth table (section 5.3.3): block 16, 8 GiB (32768 tokens
+            #      of the paper's 256 KB per token) each way, tables random and contiguous; each direction alone
+            #      ("u", end-to-end = the sum) and both at once ("b", end-to-end = the slower one)
+            def table1_cell(contiguous: bool) -> dict:
+                n = int(min(4096, (nb_gpu - 16) // 2, (nb_host - 16) // 2))
+                w4 = W.config4_sweep_case(16, contiguous, n * shape.block_bytes, nb_gpu=nb_gpu, nb_host=nb_host)
+                r4 = w4.steps[0]
+                nb4 = r4.n_out * shape.block_bytes
+                t_o = timed(lambda: pool.kv_swap_out(r4.out_gpu, r4.out_host))
+                t_i = timed(lambda: pool.kv_swap_in(r4.in_host, r4.in_gpu))
+                best = None
+                for _ in range(3):
+                    pool.kv_rotate(r4.out_gpu, r4.out_host, r4.in_host, r4.in_gpu)
+                    pool.kv_sync()
+                    s4 = pool.kv_get_stats()
+                    if best is None or s4["last_union_ms"] < best["last_union_ms"]:
+                        best = s4
+                return {"blocks_each_way": int(r4.n_out), "bytes_each_way": nb4,
+                        "d2h_u_gbs": M.gbs(nb4, t_o), "h2d_u_gbs": M.gbs(nb4, t_i), "e2e_ms_serial_u": t_o + t_i,
+                        "d2h_b_gbs": M.gbs(nb4, best["last_out_ms"]), "h2d_b_gbs": M.gbs(nb4, best["last_in_ms"]),
+                        "e2e_ms_concurrent_b": best["last_union_ms"], "both_gbs": M.gbs(2 * nb4, best["last_union_ms"]),
+                        "frac_of_probe": M.gbs(2 * nb4, best["last_union_ms"]) / p_bi_now,
+                        "path": B.PATH_NAMES[best["last_path_out"]]}
+            table1 = {"random_tables": table1_cell(False), "contiguous_tables": table1_cell(True),
+                      "paper_gh200_context": "DuplexKV 180.99 / 179.37 GB/s (b), 46.80 ms; naive 10.75 / 9.86 GB/s (u), 1556.15 ms (Table 1)"}
 
-        # ---- config 5: the serving replay at 8 requests/s under the paper's per-iteration budget of 2400
-        #      blocks; the first 200 steps that move anything, each against the 70 ms of a model step
-        try:
-            w5 = W.config5_replay(rate=8.0, nb_host=min(nb_host, 52888))
-            if w5.nb_gpu > nb_gpu:
-                raise MemoryError("device pool smaller than the replay's")
-            moving = [r5 for r5 in W.budgeted_steps(w5.steps, 2400) if r5.n_out + r5.n_in][:200]
-            ms5, blocks5 = [], []
-            for r5 in moving:
-                pool.kv_rotate(r5.out_gpu, r5.out_host, r5.in_host, r5.in_gpu)
-                pool.kv_sync()
-                ms5.append(pool.kv_get_stats()["last_union_ms"])
-                blocks5.append(r5.n_out + r5.n_in)
-            cfg5 = {"steps_timed": len(ms5), "b_xfer_blocks": 2400, "ms_median": float(np.median(ms5)),
-                    "ms_worst": float(np.max(ms5)), "blocks_median": float(np.median(blocks5)),
-                    "blocks_worst_step": int(blocks5[int(np.argmax(ms5))]),
-                    "gbs_overall": M.gbs(float(np.sum(blocks5)) * shape.block_bytes, float(np.sum(ms5))),
-                    "steps_over_70ms_model_step": int(np.sum(np.array(ms5) > 70.0)),
-                    "model_step_ms_paper": 69.82}
-        except MemoryError as e:
-            cfg5 = {"skipped": f"pools too small on this box: {e}"}
+            # ---- config 5: the serving replay at 8 requests/s under the paper's per-iteration budget of 2400
+            #      blocks; the first 200 steps that move anything, each against the 70 ms of a model step
+            try:
+                w5 = W.config5_replay(rate=8.0, nb_host=min(nb_host, 52888))
+                if w5.nb_gpu > nb_gpu:
+                    raise MemoryError("device pool smaller than the replay's")
+                moving = [r5 for r5 in W.budgeted_steps(w5.steps, 2400) if r5.n_out + r5.n_in][:200]
+                ms5, blocks5 = [], []
+                for r5 in moving:
+                    pool.kv_rotate(r5.out_gpu, r5.out_host, r5.in_host, r5.in_gpu)
+                    pool.kv_sync()
+                    ms5.append(pool.kv_get_stats()["last_union_ms"])
+                    blocks5.append(r5.n_out + r5.n_in)
+                cfg5 = {"steps_timed": len(ms5), "b_xfer_blocks": 2400, "ms_median": float(np.median(ms5)),
+                        "ms_worst": float(np.max(ms5)), "blocks_median": float(np.median(blocks5)),
+                        "blocks_worst_step": int(blocks5[int(np.argmax(ms5))]),
+                        "gbs_overall": M.gbs(float(np.sum(blocks5)) * shape.block_bytes, float(np.sum(ms5))),
+                        "steps_over_70ms_model_step": int(np.sum(np.array(ms5) > 70.0)),
+                        "model_step_ms_paper": 69.82}
+            except MemoryError as e:
+                cfg5 = {"skipped": f"pools too small on this box: {e}"}
 
-        # ---- config 3: 70B shape (5 MiB blocks, 160 planes), fragmented pool, 8 requests each way per step; a
-        #      second pool over the same device and host memory (already page-locked: no second pinning)
-        cfg3 = None
-        try:
-            s3 = W.SHAPE_70B
-            nb_gpu3 = (nb_gpu * shape.block_bytes) // s3.block_bytes
-            nb_host3 = host_bytes // s3.block_bytes
-            n3 = 12
-            w3 = W.config3_70b(nb_gpu=nb_gpu3, nb_host=nb_host3, n_steps=3 + n3)
-            pool3 = B.KVPool(s3.num_layers, s3.block_size, s3.kv_heads, s3.head_dim, nb_gpu3, nb_host3,
-                             device_pool.data_ptr(), host_base=host_base, device_id=local_rank, path=args.path,
-                             flags=args.flags, staging_bytes=args.staging_mib << 20)
-            ms3, by3 = [], []
-            for k3, r3 in enumerate(w3.steps):
-                pool3.kv_rotate(r3.out_gpu, r3.out_host, r3.in_host, r3.in_gpu)
-                pool3.kv_sync()
-                if k3 >= 3:
-                    ms3.append(pool3.kv_get_stats()["last_union_ms"])
-                    by3.append((r3.n_out + r3.n_in) * s3.block_bytes)
-            st3 = pool3.kv_get_stats()
-            g3 = [M.gbs(b, t) for b, t in zip(by3, ms3)]
-            cfg3 = {"steps_timed": len(ms3), "gpu_pool_blocks": int(nb_gpu3), "host_pool_blocks": int(nb_host3),
-                    "block_bytes": s3.block_bytes, "bytes_per_step_median": float(np.median(by3)),
-                    "ms_per_step_median": float(np.median(ms3)), "gbs_median": float(np.median(g3)),
-                    "gbs_min": float(np.min(g3)), "gbs_max": float(np.max(g3)),
-                    "frac_of_probe": float(np.median(g3)) / p_bi_now, "path": B.PATH_NAMES[st3["last_path_out"]]}
-            pool3.destroy()
-        except (MemoryError, B.KVError) as e:
-            cfg3 = {"skipped": f"not run on this box: {e}"}
+            # ---- config 3: 70B shape (5 MiB blocks, 160 planes), fragmented pool, 8 requests each way per step; a
+            #      second pool over the same device and host memory (already page-locked: no second pinning)
+            cfg3 = None
+            try:
+                s3 = W.SHAPE_70B
+                nb_gpu3 = (nb_gpu * shape.block_bytes) // s3.block_bytes
+                nb_host3 = host_bytes // s3.block_bytes
+                n3 = 12
+                w3 = W.config3_70b(nb_gpu=nb_gpu3, nb_host=nb_host3, n_steps=3 + n3)
+                pool3 = B.KVPool(s3.num_layers, s3.block_size, s3.kv_heads, s3.head_dim, nb_gpu3, nb_host3,
+                                 device_pool.data_ptr(), host_base=host_base, device_id=local_rank, path=args.path,
+                                 flags=args.flags, staging_bytes=args.staging_mib << 20)
+                ms3, by3 = [], []
+                for k3, r3 in enumerate(w3.steps):
+                    pool3.kv_rotate(r3.out_gpu, r3.out_host, r3.in_host, r3.in_gpu)
+                    pool3.kv_sync()
+                    if k3 >= 3:
+                        ms3.append(pool3.kv_get_stats()["last_union_ms"])
+                        by3.append((r3.n_out + r3.n_in) * s3.block_bytes)
+                st3 = pool3.kv_get_stats()
+                g3 = [M.gbs(b, t) for b, t in zip(by3, ms3)]
+                cfg3 = {"steps_timed": len(ms3), "gpu_pool_blocks": int(nb_gpu3), "host_pool_blocks": int(nb_host3),
+                        "block_bytes": s3.block_bytes, "bytes_per_step_median": float(np.median(by3)),
+                        "ms_per_step_median": float(np.median(ms3)), "gbs_median": float(np.median(g3)),
+                        "gbs_min": float(np.min(g3)), "gbs_max": float(np.max(g3)),
+                        "frac_of_probe": float(np.median(g3)) / p_bi_now, "path": B.PATH_NAMES[st3["last_path_out"]]}
+                pool3.destroy()
+            except (MemoryError, B.KVError) as e:
+                cfg3 = {"skipped": f"not run on this box: {e}"}
 
         extra = {"paths": paths, "singles": singles, "lat_us": lat_us, "lat_blocks": lat_blocks, "leg": leg,
                  "leg_bytes": leg_bytes, "probe2": probe2, "contiguous_host": contiguous_host, "table": tb,
@@ -616,6 +618,7 @@ def main() -> None:
     ap.add_argument("--flags", type=int, default=0, help="KV_FLAG_* bits")
     ap.add_argument("--ctas", type=int, default=0, help="CTAs per direction (0 = default)")
     ap.add_argument("--staging-mib", type=int, default=0, help="per-direction staging of the staged path (0 = library default)")
+    ap.add_argument("--link-variant", type=int, default=0, help="shape of the zero-copy kernels' transfers (0, 1, 2)")
     ap.add_argument("--quick", action="store_true", help="skip the per-segment comparator path")
     ap.add_argument("--trace", default=None, help="write a Chrome-trace JSON of the timed steps' two directions here")
     ap.add_argument("--small", action="store_true",

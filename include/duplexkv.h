@@ -58,10 +58,10 @@ extern "C" {
 #define KV_DEV_BLOCK_FIRST    1     /* [block][layer][K|V]...: the paper's redesigned storage order      */
 
 /* transfer paths (how the host link is driven) */
-#define KV_PATH_AUTO          0     /* per call.  Calls bound by fixed costs: CE2D when the call moves 8 MiB
-                                       or less per direction, ZEROCOPY up to 24 MiB.  Larger calls: STAGED
-                                       when the copy-engine transfers the call needs would average 3 MiB
-                                       or more, else ZEROCOPY (see kv_path_for)                          */
+#define KV_PATH_AUTO          0     /* per call.  Calls bound by fixed costs, 32 MiB or less per direction:
+                                       CE2D (blocks under 2 MiB: CE2D up to 8 MiB, ZEROCOPY above).  Larger
+                                       calls: STAGED when the copy-engine transfers the call needs would
+                                       average 3 MiB or more, else ZEROCOPY (see kv_path_for)            */
 #define KV_PATH_ZEROCOPY      1     /* SM kernels read/write mapped pinned host memory directly          */
 #define KV_PATH_STAGED        2     /* pack kernel -> contiguous HBM staging -> copy engine (and reverse)*/
 #define KV_PATH_CE2D          3     /* one strided 2-D copy-engine transfer per block, no kernel         */
@@ -76,6 +76,11 @@ extern "C" {
                                        between the directions, on the out stream.  Without the flag this
                                        is done only for short lists (64 blocks or fewer each way) on an
                                        idle pool, where it saves a launch; longer ones use two streams   */
+#define KV_FLAG_DEBUG_BOUNDS    16  /* the kernels compare every block id with its pool's size before they form an
+                                       address from it; an id out of bounds is skipped (none of its bytes is
+                                       touched), recorded in the status word, and kv_sync returns KV_ERR_RANGE.
+                                       The host-side checks already refuse such ids before any launch; this
+                                       guards the path from the id ring to the kernel (a debugging aid)   */
 #define KV_FLAG_TIME_KERNELS    8   /* bracket every HBM-to-HBM gather / scatter kernel (STAGED pack / unpack,
                                        kv_gather_blocks, kv_scatter_blocks) with events on its own stream;
                                        kv_sync adds their durations to the timed_* statistics            */
@@ -98,14 +103,18 @@ typedef struct {
     int32_t device_id;
     void   *stream_out;     /* cudaStream_t or NULL (library creates a non-blocking stream)               */
     void   *stream_in;      /* likewise; must differ from stream_out for the directions to overlap        */
-    int32_t path;           /* KV_PATH_* of the swap-out direction, and of swap-in unless path_in is set  */
+    int32_t path;           /* KV_PATH_* of the swap-out direction, and of swap-in unless path_in is set.
+                               The environment overrides it: DUPLEXKV_PATH = auto | zerocopy | staged |
+                               ce2d | naive (both directions); likewise DUPLEXKV_SMS_OUT / DUPLEXKV_SMS_IN
+                               for ctas_out / ctas_in.  A value that does not parse fails the create       */
     int32_t flags;          /* KV_FLAG_*                                                                  */
     int32_t ctas_out;       /* CTAs of the zero-copy swap-out kernel, 0 = 64                              */
     int32_t ctas_in;        /* CTAs of the swap-in kernel, 0 = default                                    */
     int64_t staging_bytes;  /* per-direction HBM staging of the STAGED path (two halves used as a double
-                               buffer, allocated at the first staged call); 0 = 2 GiB or a sixteenth of the
-                               device pool, whichever is smaller; at least 2*BLK.  Larger halves mean fewer
-                               and longer pack / unpack launches                                          */
+                               buffer, allocated at the first staged call); 0 = a sixteenth of the device
+                               pool, but at most 2 GiB and at least 128 MiB (or the pool's own size if that
+                               is smaller); never less than 2*BLK.  Larger halves mean fewer and longer
+                               pack / unpack launches                                                     */
     int32_t path_in;        /* KV_PATH_* of the swap-in direction; KV_PATH_AUTO (0) = same as `path`      */
     int32_t ce_streams;     /* streams per direction that the copy-engine paths spread their transfers
                                over (1..4), 0 = 1                                                         */
@@ -113,7 +122,10 @@ typedef struct {
                                4.3.2 in which all layers of a device block are contiguous (a consumer of
                                the pool then strides by BLK between blocks).  kv_gather_blocks_static
                                reads layer-first pools only                                               */
-    int32_t pad_;
+    int32_t link_variant;   /* shape of the zero-copy kernels' transfers (a measurement knob; 0 is the default and
+                               the quickest found): bulk kernel: 0 = 8 KiB copies, 8-stage ring; 1 = 32 KiB
+                               copies, 4 stages; 2 = 64 KiB copies, 3 stages.  With KV_FLAG_LDST_KERNEL:
+                               1 = 32-byte instead of 16-byte vectors per thread                          */
 } kv_pool_config_t;
 
 typedef struct {
@@ -137,6 +149,7 @@ typedef struct {
                                           CTA end (%globaltimer), i.e. without the wait for the launch     */
     double  last_in_offset_ms;         /* latest kv_rotate: start of its swap-in window minus start of its
                                           swap-out window (with last_out_ms and last_in_ms: the timeline)  */
+    int64_t requests_out, requests_in; /* requests that kv_rotate_req calls carried, per direction          */
 } kv_stats_t;
 
 typedef struct {
@@ -183,6 +196,20 @@ int32_t kv_swap_in(kv_pool_t *pool, const int32_t *host_ids, const int32_t *gpu_
 int32_t kv_rotate(kv_pool_t *pool,
                   const int32_t *out_gpu, const int32_t *out_host, int64_t n_out,
                   const int32_t *in_host, const int32_t *in_gpu, int64_t n_in);
+
+/*
+ * kv_rotate with the request boundaries of its lists, for per-request statistics only: request r of the
+ * swap-out owns list entries out_req_offsets[r] .. out_req_offsets[r+1]-1 (HOST arrays of n_out_req + 1
+ * and n_in_req + 1 non-decreasing offsets, first 0, last n_out / n_in; a direction without blocks takes
+ * NULL and 0).  Moves exactly what kv_rotate would and adds the request counts to the statistics, so that
+ * time and bytes per request can be had from kv_get_stats.  Bad offsets: KV_ERR_INVALID_ARG, nothing
+ * moves.  (The paper rotates whole requests, section 4.2; a request is a contiguous run of the lists.)
+ */
+int32_t kv_rotate_req(kv_pool_t *pool,
+                      const int32_t *out_gpu, const int32_t *out_host, int64_t n_out,
+                      const int64_t *out_req_offsets, int64_t n_out_req,
+                      const int32_t *in_host, const int32_t *in_gpu, int64_t n_in,
+                      const int64_t *in_req_offsets, int64_t n_in_req);
 
 /*
  * What copy-engine transfers the STAGED path would make for one direction of a call (no pool, no GPU):
@@ -344,6 +371,23 @@ int32_t kv_pool_shape(kv_pool_t *pool, kv_pool_shape_t *out);
  * rotation runs beside model execution and nobody wants a host-side kv_sync.
  */
 int32_t kv_stream_wait(kv_pool_t *pool, void *stream, int32_t directions);
+
+/*
+ * The event that completes with the latest call issued so far in `direction` (0 = swap-outs, 1 = swap-ins):
+ * *event receives a cudaEvent_t owned by the pool, or NULL when the direction has seen no call yet.  It
+ * stays that call's event until eight further calls of the direction have been issued, and dies with the
+ * pool.  For cudaStreamWaitEvent / cudaEventQuery / cudaEventSynchronize by whoever schedules the model's
+ * kernels: the completion signal of the paper's cross-iteration pipeline (section 4.3.2), where iteration
+ * t computes while the transfers of t+1 are in flight.  kv_stream_wait is the same thing done in one call.
+ */
+int32_t kv_completion_event(kv_pool_t *pool, int32_t direction, void **event);
+
+/* Waits for outstanding work, then sets the CTAs of the zero-copy kernels per direction (0 = the default,
+ * 64).  How many SMs a rotation may occupy beside model execution is a sizing decision of the caller. */
+int32_t kv_pool_set_ctas(kv_pool_t *pool, int32_t ctas_out, int32_t ctas_in);
+
+/* The predicate behind KV_FLAG_DEBUG_BOUNDS as a host function: 1 when both ids lie inside their pools. */
+int32_t kv_debug_pair_in_bounds(int32_t src_id, int32_t dst_id, int32_t src_blocks, int32_t dst_blocks);
 
 /* Calls issued and calls known to have completed, per direction (a non-blocking look at the pool's
  * end events).  Any pointer may be NULL.  kv_gather_blocks / kv_scatter_blocks count as calls of the

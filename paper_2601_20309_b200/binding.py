@@ -41,6 +41,7 @@ KV_FLAG_ALLOW_OVERLAP = 1
 KV_FLAG_LDST_KERNEL = 2
 KV_FLAG_FUSED_ROTATE = 4
 KV_FLAG_TIME_KERNELS = 8
+KV_FLAG_DEBUG_BOUNDS = 16
 
 
 class kv_pool_config_t(C.Structure):
@@ -50,7 +51,7 @@ class kv_pool_config_t(C.Structure):
                 ("device_id", C.c_int32), ("stream_out", C.c_void_p), ("stream_in", C.c_void_p),
                 ("path", C.c_int32), ("flags", C.c_int32), ("ctas_out", C.c_int32), ("ctas_in", C.c_int32),
                 ("staging_bytes", C.c_int64), ("path_in", C.c_int32), ("ce_streams", C.c_int32),
-                ("device_layout", C.c_int32), ("pad_", C.c_int32)]
+                ("device_layout", C.c_int32), ("link_variant", C.c_int32)]
 
 
 class kv_stats_t(C.Structure):
@@ -60,7 +61,8 @@ class kv_stats_t(C.Structure):
                 ("last_path_out", C.c_int32), ("last_path_in", C.c_int32),
                 ("device_status", C.c_uint32), ("pad_", C.c_int32),
                 ("timed_kernel_ms", C.c_double), ("timed_kernel_bytes", C.c_int64), ("timed_kernels", C.c_int64),
-                ("timed_kernel_exec_ms", C.c_double), ("last_in_offset_ms", C.c_double)]
+                ("timed_kernel_exec_ms", C.c_double), ("last_in_offset_ms", C.c_double),
+                ("requests_out", C.c_int64), ("requests_in", C.c_int64)]
 
 
 class kv_link_probe_t(C.Structure):
@@ -105,7 +107,8 @@ EXPORTS = ["kv_pool_create", "kv_pool_destroy", "kv_pool_set_path", "kv_swap_out
            "kv_table_create", "kv_table_create_dry", "kv_table_destroy", "kv_table_last_error", "kv_req_add",
            "kv_req_append", "kv_eager_rotate", "kv_req_rotate", "kv_req_preempt", "kv_req_resume", "kv_req_finish",
            "kv_req_info", "kv_req_blocks", "kv_table_get_stats", "kv_table_fail_pool_call",
-           "kv_pool_set_wait_limit", "kv_pool_set_call_timing"]
+           "kv_pool_set_wait_limit", "kv_pool_set_call_timing", "kv_completion_event", "kv_pool_set_ctas",
+           "kv_debug_pair_in_bounds", "kv_rotate_req"]
 
 _lib = None
 
@@ -184,6 +187,14 @@ def lib() -> C.CDLL:
     L.kv_req_blocks.argtypes = [vp, i64, i32p, i32p, C.POINTER(C.c_uint8), i64]
     L.kv_table_get_stats.restype = C.c_int32
     L.kv_table_get_stats.argtypes = [vp, C.POINTER(kv_table_stats_t)]
+    L.kv_completion_event.restype = C.c_int32
+    L.kv_completion_event.argtypes = [vp, C.c_int32, C.POINTER(vp)]
+    L.kv_pool_set_ctas.restype = C.c_int32
+    L.kv_pool_set_ctas.argtypes = [vp, C.c_int32, C.c_int32]
+    L.kv_debug_pair_in_bounds.restype = C.c_int32
+    L.kv_debug_pair_in_bounds.argtypes = [C.c_int32] * 4
+    L.kv_rotate_req.restype = C.c_int32
+    L.kv_rotate_req.argtypes = [vp, i32p, i32p, i64, C.POINTER(C.c_int64), i64, i32p, i32p, i64, C.POINTER(C.c_int64), i64]
     L.kv_pool_set_call_timing.restype = C.c_int32
     L.kv_pool_set_call_timing.argtypes = [vp, C.c_int32]
     L.kv_pool_set_wait_limit.restype = C.c_int32
@@ -219,6 +230,10 @@ def kv_seg_bytes(block_size: int, kv_heads: int, head_dim: int) -> int:
 
 def kv_blk_bytes(num_layers: int, block_size: int, kv_heads: int, head_dim: int) -> int:
     return lib().kv_blk_bytes(num_layers, block_size, kv_heads, head_dim)
+
+
+def kv_debug_pair_in_bounds(src_id: int, dst_id: int, src_blocks: int, dst_blocks: int) -> bool:
+    return bool(lib().kv_debug_pair_in_bounds(src_id, dst_id, src_blocks, dst_blocks))
 
 
 def kv_path_for(blk_bytes: int) -> int:
@@ -285,11 +300,11 @@ class KVPool:
                  device_id: int = 0, stream_out: Optional[int] = None, stream_in: Optional[int] = None,
                  path: int = KV_PATH_AUTO, flags: int = 0, ctas_out: int = 0, ctas_in: int = 0,
                  staging_bytes: int = 0, path_in: int = KV_PATH_AUTO, ce_streams: int = 0,
-                 device_layout: int = KV_DEV_LAYER_FIRST):
+                 device_layout: int = KV_DEV_LAYER_FIRST, link_variant: int = 0):
         self.cfg = kv_pool_config_t(num_layers, block_size, kv_heads, head_dim, num_gpu_blocks,
                                     num_host_blocks, device_base, host_base, host_layout, device_id,
                                     stream_out, stream_in, path, flags, ctas_out, ctas_in, staging_bytes,
-                                    path_in, ce_streams, device_layout, 0)
+                                    path_in, ce_streams, device_layout, link_variant)
         self._h = C.c_void_p()
         rc = lib().kv_pool_create(C.byref(self.cfg), C.byref(self._h))
         if rc != KV_OK:
@@ -350,6 +365,27 @@ class KVPool:
 
     def kv_pool_set_path(self, path_out: int, path_in: int, check: bool = True) -> int:
         return self._ret(lib().kv_pool_set_path(self._h, path_out, path_in), check)
+
+    def kv_completion_event(self, direction: int) -> Optional[int]:
+        """The pool-owned ``cudaEvent_t`` (as an integer handle) of the latest call of ``direction``, or None."""
+        ev = C.c_void_p()
+        self._ret(lib().kv_completion_event(self._h, direction, C.byref(ev)), True)
+        return ev.value
+
+    def kv_pool_set_ctas(self, ctas_out: int, ctas_in: int, check: bool = True) -> int:
+        return self._ret(lib().kv_pool_set_ctas(self._h, ctas_out, ctas_in), check)
+
+    def kv_rotate_req(self, out_gpu, out_host, out_req_offsets, in_host, in_gpu, in_req_offsets, check: bool = True) -> int:
+        og, ogp = _ids(out_gpu)
+        oh, ohp = _ids(out_host)
+        ih, ihp = _ids(in_host)
+        ig, igp = _ids(in_gpu)
+        oo = np.ascontiguousarray(np.asarray(out_req_offsets, dtype=np.int64))
+        io = np.ascontiguousarray(np.asarray(in_req_offsets, dtype=np.int64))
+        i64p = C.POINTER(C.c_int64)
+        return self._ret(lib().kv_rotate_req(self._h, ogp, ohp, len(og), oo.ctypes.data_as(i64p) if len(oo) else None,
+                                             max(0, len(oo) - 1), ihp, igp, len(ig),
+                                             io.ctypes.data_as(i64p) if len(io) else None, max(0, len(io) - 1)), check)
 
     def kv_pool_set_call_timing(self, on: bool, check: bool = True) -> int:
         return self._ret(lib().kv_pool_set_call_timing(self._h, int(on)), check)

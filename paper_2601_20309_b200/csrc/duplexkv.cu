@@ -12,6 +12,7 @@
 #include <algorithm>
 #include <chrono>
 #include <cstdio>
+#include <cstdlib>
 #include <cstring>
 #include <new>
 #include <vector>
@@ -22,12 +23,15 @@ constexpr int KV_SLOTS = 8;            // descriptor / event ring depth per dire
 constexpr int KV_MAX_CE_STREAMS = 4;
 constexpr int64_t KV_AUTO_MIN_TRANSFER = 3ll << 20;   // AUTO: staged when its transfers average 3 MiB or more
 // AUTO, calls bound by fixed costs rather than by the link (measured on 2 MiB blocks, scattered ids, call to
-// completion): up to 8 MiB per direction one copy-engine transfer per block is quickest (73 / 117 / 232 us for
-// 1 / 2 / 4 blocks each way against 92 / 148 / 251 us for the zero-copy kernels, whose duplex rate is lower);
-// up to 24 MiB the zero-copy kernels are (462 us at 8 blocks against 470 and 496); from 32 MiB on the staged
-// pipeline is ahead and the transfer-size rule below decides.
-constexpr int64_t KV_AUTO_TINY_BYTES = 8ll << 20;
-constexpr int64_t KV_AUTO_SMALL_BYTES = 24ll << 20;
+// completion, two runs): one copy-engine transfer per block is the quickest or within 1.5 % of it up to 16
+// blocks each way (64 / 109 / 216 / 420-470 / 826-858 us for 1 / 2 / 4 / 8 / 16 blocks against 86 / 142 /
+// 247 / 455 / 882-900 us for the zero-copy kernels and 93 / 145 / 239 / 494 / 849-860 us staged); from 32
+// blocks on the staged pipeline is ahead and the transfer-size rule decides.  One transfer per block needs
+// blocks of 2 MiB or more to reach the kernels' rate; smaller blocks take that path only up to 8 MiB and the
+// zero-copy kernels above that.
+constexpr int64_t KV_AUTO_TINY_BYTES = 32ll << 20;
+constexpr int64_t KV_AUTO_TINY_BYTES_SMALL_BLOCKS = 8ll << 20;
+constexpr int64_t KV_AUTO_SMALL_BYTES = 32ll << 20;
 constexpr int64_t KV_MERGE_MIN_MEAN_RUN = 8;
 constexpr int64_t KV_PLAN_CHUNKS = 4;                 // STAGED: a call that fits one staging half is still cut into about this many chunks          // STAGED: merge runs of host ids when they average 8 blocks or more
 constexpr int BULK_STAGE = 16384;      // bytes per shared-memory stage of the bulk kernel
@@ -38,9 +42,13 @@ constexpr int BULK_AHEAD = 5;          // loads in flight ahead of the stores
 constexpr int LINK_STAGE = 8192;
 constexpr int LINK_NS = 8;
 constexpr int LINK_AHEAD = 6;
+// other shapes of the same ring for the link (kv_pool_config_t.link_variant 1 and 2): fewer, larger bulk copies
+constexpr int LINK1_STAGE = 32768, LINK1_NS = 4, LINK1_AHEAD = 2;
+constexpr int LINK2_STAGE = 65536, LINK2_NS = 3, LINK2_AHEAD = 1;
 constexpr int LDST_THREADS = 512;
 constexpr int LDST_UNROLL = 4;         // 512 threads * 4 * 16 B = 32 KiB per item
 constexpr int LDST_CHUNK = LDST_THREADS * LDST_UNROLL * 16;
+constexpr int LDST32_UNROLL = 2;       // 512 threads * 2 * 32 B = 32 KiB per item
 
 thread_local char g_err[256] = "";
 
@@ -179,9 +187,23 @@ KvSide packed_side(const kv_pool *p, const void *base)
 
 bool use_ldst(const kv_pool *p) { return (p->cfg.flags & KV_FLAG_LDST_KERNEL) != 0; }
 
+// which shape of the bulk kernel's ring a zero-copy launch uses
+int link_stage(const kv_pool *p)
+{
+    return p->cfg.link_variant == 1 ? LINK1_STAGE : (p->cfg.link_variant == 2 ? LINK2_STAGE : LINK_STAGE);
+}
+
+// 32-byte vectors in the load/store kernel: zero-copy launches of a pool that asks for them, when every
+// address they form is 32-byte aligned
+bool ldst32(const kv_pool *p, bool link)
+{
+    return link && use_ldst(p) && p->cfg.link_variant == 1 && p->seg % 32 == 0 && ((uintptr_t)p->dev & 31) == 0 &&
+           ((uintptr_t)p->host_dev & 31) == 0;
+}
+
 void fill_geometry(const kv_pool *p, KvJob &job, bool link = false)
 {
-    const int max_chunk = use_ldst(p) ? LDST_CHUNK : (link ? LINK_STAGE : BULK_STAGE);
+    const int max_chunk = use_ldst(p) ? LDST_CHUNK : (link ? link_stage(p) : BULK_STAGE);
     job.planes = p->planes;
     job.seg = (int)p->seg;
     job.chunk = (int)std::min<int64_t>(p->seg, max_chunk);
@@ -189,6 +211,7 @@ void fill_geometry(const kv_pool *p, KvJob &job, bool link = false)
     job.status = p->status_dev;
     job.wait_polls = p->wait_polls;
     job.wait_ns = p->wait_ns;
+    job.check_ids = (p->cfg.flags & KV_FLAG_DEBUG_BOUNDS) ? 1 : 0;
     job.t_first = job.t_last = nullptr;
 }
 
@@ -203,7 +226,12 @@ cudaError_t launch_job(kv_pool *p, const KvJob &job, cudaStream_t stream, bool l
     const int grid = job.dir[0].ctas + job.dir[1].ctas;
     if (grid <= 0) return cudaSuccess;
     if (use_ldst(p)) {
-        kv_copy_ldst<LDST_THREADS, LDST_UNROLL><<<grid, LDST_THREADS, 0, stream>>>(job);
+        if (ldst32(p, link)) kv_copy_ldst<LDST_THREADS, LDST32_UNROLL, 32><<<grid, LDST_THREADS, 0, stream>>>(job);
+        else kv_copy_ldst<LDST_THREADS, LDST_UNROLL, 16><<<grid, LDST_THREADS, 0, stream>>>(job);
+    } else if (link && p->cfg.link_variant == 1) {
+        kv_copy_bulk<LINK1_STAGE, LINK1_NS, LINK1_AHEAD><<<grid, 32, LINK1_STAGE * LINK1_NS, stream>>>(job);
+    } else if (link && p->cfg.link_variant == 2) {
+        kv_copy_bulk<LINK2_STAGE, LINK2_NS, LINK2_AHEAD><<<grid, 32, LINK2_STAGE * LINK2_NS, stream>>>(job);
     } else if (link) {
         kv_copy_bulk<LINK_STAGE, LINK_NS, LINK_AHEAD><<<grid, 32, LINK_STAGE * LINK_NS, stream>>>(job);
     } else {
@@ -548,7 +576,11 @@ int32_t begin_dir(kv_pool *p, DirCall &c, cudaEvent_t wait_for)
         if (c.n > KV_INLINE_PAIRS)
             KV_CUDA(p, cudaMemcpyAsync(c.pairs_dev, c.pairs_host, (size_t)c.n * sizeof(int2), cudaMemcpyHostToDevice, s.stream));
     } else if (c.path == KV_PATH_STAGED) {
-        KV_CUDA(p, cudaMemcpyAsync(c.aux_dev, c.aux_host, (size_t)c.n * sizeof(int2), cudaMemcpyHostToDevice, s.stream));
+        // chunks of KV_INLINE_PAIRS blocks or fewer carry their ids in the launch parameters (ce_issue_some)
+        bool ids_on_device = false;
+        for (const CeChunk &ch : s.chunks) ids_on_device = ids_on_device || ch.hi - ch.lo > KV_INLINE_PAIRS;
+        if (ids_on_device)
+            KV_CUDA(p, cudaMemcpyAsync(c.aux_dev, c.aux_host, (size_t)c.n * sizeof(int2), cudaMemcpyHostToDevice, s.stream));
         // the kernel stream starts after everything issued so far on this direction
         KV_CUDA(p, cudaEventRecord(s.kfork_ev, s.stream));
         KV_CUDA(p, cudaStreamWaitEvent(s.kstream, s.kfork_ev, 0));
@@ -596,6 +628,8 @@ void zerocopy_dir(kv_pool *p, const DirCall &c, KvJob &job, int k)
     d.dst = (c.d == 0) ? host_side(p) : device_side(p);
     d.n = (int)c.n;
     d.ctas = 0;
+    d.src_blocks = (int)(c.d == 0 ? p->cfg.num_gpu_blocks : p->cfg.num_host_blocks);
+    d.dst_blocks = (int)(c.d == 0 ? p->cfg.num_host_blocks : p->cfg.num_gpu_blocks);
     if (c.n <= KV_INLINE_PAIRS) {
         d.pairs = nullptr;
         for (int64_t i = 0; i < c.n; ++i)
@@ -675,6 +709,13 @@ int32_t ce_issue_some(kv_pool *p, DirCall &c, int budget, bool &finished)
         kd.dst = (c.d == 0) ? st : device_side(p);
         kd.pairs = c.aux_dev + ch.lo;
         kd.n = (int)(ch.hi - ch.lo);
+        if (kd.n <= KV_INLINE_PAIRS) {
+            kd.pairs = nullptr;
+            for (int q = 0; q < kd.n; ++q) job.inl[0][q] = c.aux_host[ch.lo + q];
+        }
+        // staging-side "ids" are positions of the sorted list, below ch.hi
+        kd.src_blocks = (int)(c.d == 0 ? p->cfg.num_gpu_blocks : ch.hi);
+        kd.dst_blocks = (int)(c.d == 0 ? ch.hi : p->cfg.num_gpu_blocks);
         kd.ctas = clamp_ctas(job, kd, p->sm_count);
         if (!c.chunk_open) {
             if (c.d == 0) {
@@ -772,8 +813,8 @@ int32_t run_calls(kv_pool *p, DirCall *calls, int ncalls, const bool *wait_other
             wait_ev[k] = o.ev_end[o.issued % KV_SLOTS];
         }
     // KV_PATH_AUTO is settled per call.  A call that moves little is bound by its fixed costs, not by the
-    // link: up to KV_AUTO_TINY_BYTES per direction it goes as one copy-engine transfer per block, up to
-    // KV_AUTO_SMALL_BYTES to the zero-copy kernels (one launch, no staging pipeline).  Otherwise the staged
+    // link: up to KV_AUTO_TINY_BYTES per direction (less for blocks under 2 MiB) it goes as one copy-engine
+    // transfer per block, up to KV_AUTO_SMALL_BYTES to the zero-copy kernels (one launch, no staging pipeline).  Otherwise the staged
     // transfers are planned first (cheap: a sort of the ids) and the staged path is taken when its transfers
     // would carry KV_AUTO_MIN_TRANSFER bytes or more on average, the zero-copy kernels when not.  Both
     // directions of a rotate take the same path (a kernel on one direction starves the copy engine on the
@@ -785,7 +826,7 @@ int32_t run_calls(kv_pool *p, DirCall *calls, int ncalls, const bool *wait_other
             if (calls[k].path == KV_PATH_AUTO) largest = std::max(largest, calls[k].n * p->blk);
         }
         int chosen;
-        if (largest <= KV_AUTO_TINY_BYTES) {
+        if (largest <= (p->blk >= (2ll << 20) ? KV_AUTO_TINY_BYTES : KV_AUTO_TINY_BYTES_SMALL_BLOCKS)) {
             chosen = KV_PATH_CE2D;
         } else if (largest <= KV_AUTO_SMALL_BYTES) {
             chosen = KV_PATH_ZEROCOPY;
@@ -952,9 +993,33 @@ int32_t kv_pool_create(const kv_pool_config_t *cfg, kv_pool_t **out)
     if (cfg->path < KV_PATH_AUTO || cfg->path > KV_PATH_NAIVE || cfg->path_in < KV_PATH_AUTO || cfg->path_in > KV_PATH_NAIVE)
         return fail(nullptr, KV_ERR_INVALID_ARG, "unknown path");
     if (cfg->ctas_out < 0 || cfg->ctas_in < 0 || cfg->staging_bytes < 0 || cfg->ce_streams < 0 ||
-        cfg->ce_streams > KV_MAX_CE_STREAMS)
+        cfg->ce_streams > KV_MAX_CE_STREAMS || cfg->link_variant < 0 || cfg->link_variant > 2)
         return fail(nullptr, KV_ERR_INVALID_ARG, "tuning value out of range");
 
+    // environment overrides of the path and of the zero-copy CTA counts (for trying settings on a program
+    // that cannot be rebuilt); a value that does not parse is an error, not ignored
+    kv_pool_config_t eff = *cfg;
+    {
+        static const char *names[] = {"auto", "zerocopy", "staged", "ce2d", "naive"};
+        if (const char *v = getenv("DUPLEXKV_PATH")) {
+            int found = -1;
+            for (int k = 0; k < 5; ++k)
+                if (!strcmp(v, names[k])) found = k;
+            if (found < 0) return fail(nullptr, KV_ERR_INVALID_ARG, "DUPLEXKV_PATH must be auto, zerocopy, staged, ce2d or naive");
+            eff.path = found;
+            eff.path_in = KV_PATH_AUTO;        // "same as path"
+        }
+        const char *keys[2] = {"DUPLEXKV_SMS_OUT", "DUPLEXKV_SMS_IN"};
+        int32_t *dst[2] = {&eff.ctas_out, &eff.ctas_in};
+        for (int k = 0; k < 2; ++k)
+            if (const char *v = getenv(keys[k])) {
+                char *end = nullptr;
+                const long x = strtol(v, &end, 10);
+                if (end == v || *end || x < 0 || x > 65535) return fail(nullptr, KV_ERR_INVALID_ARG, "DUPLEXKV_SMS_OUT / DUPLEXKV_SMS_IN must be a CTA count");
+                *dst[k] = (int32_t)x;
+            }
+    }
+    cfg = &eff;
     KV_CUDA(nullptr, cudaSetDevice(cfg->device_id));
     kv_pool *p = new (std::nothrow) kv_pool();
     if (!p) return fail(nullptr, KV_ERR_NOMEM, "out of host memory");
@@ -966,8 +1031,13 @@ int32_t kv_pool_create(const kv_pool_config_t *cfg, kv_pool_t **out)
     p->dev = (uint8_t *)cfg->device_base;
     p->err[0] = 0;
     memset(&p->stats, 0, sizeof(p->stats));
-    // default staging: 2 GiB per direction, but no more than a sixteenth of the device pool
-    if (p->cfg.staging_bytes == 0) p->cfg.staging_bytes = std::min<int64_t>(2ll << 30, cfg->num_gpu_blocks * blk / 16);
+    // default staging: 2 GiB per direction, but no more than a sixteenth of the device pool -- or 128 MiB (the
+    // whole pool's size if that is less) when the pool is small: halves of a few blocks would turn every
+    // call into a chain of tiny chunks with an event hand-off between each
+    if (p->cfg.staging_bytes == 0) {
+        const int64_t pool_bytes = cfg->num_gpu_blocks * blk;
+        p->cfg.staging_bytes = std::min<int64_t>(2ll << 30, std::max<int64_t>(pool_bytes / 16, std::min<int64_t>(pool_bytes, 128ll << 20)));
+    }
     if (p->cfg.staging_bytes < 2 * blk) p->cfg.staging_bytes = 2 * blk;
 
 #define KV_CREATE_CUDA(expr)                                   \
@@ -988,17 +1058,25 @@ int32_t kv_pool_create(const kv_pool_config_t *cfg, kv_pool_t **out)
     const size_t host_bytes = (size_t)cfg->num_host_blocks * (size_t)blk;
     if (cfg->host_base) {
         p->host = (uint8_t *)cfg->host_base;
-        cudaError_t e = cudaHostRegister(p->host, host_bytes, cudaHostRegisterMapped | cudaHostRegisterPortable);
-        if (e == cudaErrorHostMemoryAlreadyRegistered) {
-            // page-locked already (by the caller, or it is another pool's host memory): used as it is and
-            // left page-locked at destroy
-            (void)cudaGetLastError();
-        } else if (e != cudaSuccess) {
-            (void)cudaGetLastError();
-            int32_t rc = fail(nullptr, KV_ERR_NOMEM, "cudaHostRegister of host_base failed");
-            kv_pool_destroy(p);
-            return rc;
-        } else {
+        // Memory that CUDA knows as page-locked already (allocated by cudaHostAlloc, registered by the caller,
+        // or the host memory of another pool) is used as it is and left page-locked at destroy; the first
+        // and the last byte are looked up.
+        auto pinned = [](const void *q) {
+            cudaPointerAttributes a;
+            if (cudaPointerGetAttributes(&a, q) != cudaSuccess) {
+                (void)cudaGetLastError();
+                return false;
+            }
+            return a.type == cudaMemoryTypeHost;
+        };
+        if (!(pinned(p->host) && pinned(p->host + host_bytes - 1))) {
+            cudaError_t e = cudaHostRegister(p->host, host_bytes, cudaHostRegisterMapped | cudaHostRegisterPortable);
+            if (e != cudaSuccess) {
+                (void)cudaGetLastError();
+                int32_t rc = fail(nullptr, KV_ERR_NOMEM, "cudaHostRegister of host_base failed");
+                kv_pool_destroy(p);
+                return rc;
+            }
             p->registered_host = true;
         }
     } else {
@@ -1055,6 +1133,10 @@ int32_t kv_pool_create(const kv_pool_config_t *cfg, kv_pool_t **out)
                                         cudaFuncAttributeMaxDynamicSharedMemorySize, BULK_STAGE * BULK_NS));
     KV_CREATE_CUDA(cudaFuncSetAttribute(kv_copy_bulk<LINK_STAGE, LINK_NS, LINK_AHEAD>,
                                         cudaFuncAttributeMaxDynamicSharedMemorySize, LINK_STAGE * LINK_NS));
+    KV_CREATE_CUDA(cudaFuncSetAttribute(kv_copy_bulk<LINK1_STAGE, LINK1_NS, LINK1_AHEAD>,
+                                        cudaFuncAttributeMaxDynamicSharedMemorySize, LINK1_STAGE * LINK1_NS));
+    KV_CREATE_CUDA(cudaFuncSetAttribute(kv_copy_bulk<LINK2_STAGE, LINK2_NS, LINK2_AHEAD>,
+                                        cudaFuncAttributeMaxDynamicSharedMemorySize, LINK2_STAGE * LINK2_NS));
 #undef KV_CREATE_CUDA
 
     try {
@@ -1330,6 +1412,9 @@ int32_t kv_sync(kv_pool_t *p)
     if (st & KV_DEV_TIMEOUT) {
         if (p->sticky == KV_OK) p->sticky = KV_ERR_TIMEOUT;
         snprintf(p->err, 256, "a device-side wait ran out (status 0x%x)", st);
+    } else if (st & KV_DEV_BAD_ID) {
+        if (p->sticky == KV_OK) p->sticky = KV_ERR_RANGE;
+        snprintf(p->err, 256, "a kernel met a block id outside its pool and skipped it (status 0x%x)", st);
     }
     return p->sticky;
 }
@@ -1375,6 +1460,8 @@ static int32_t device_leg(kv_pool_t *p, const int32_t *gpu_ids, int64_t n, const
     kd.dst = (d == 0) ? packed_side(p, buf) : device_side(p);
     kd.pairs = pd;
     kd.n = (int)n;
+    kd.src_blocks = (int)(d == 0 ? p->cfg.num_gpu_blocks : n);
+    kd.dst_blocks = (int)(d == 0 ? n : p->cfg.num_gpu_blocks);
     const int want = (d == 0 ? p->cfg.ctas_out : p->cfg.ctas_in);
     kd.ctas = clamp_ctas(job, kd, want > 0 ? want : p->sm_count);
     KV_CUDA(p, launch_timed(p, s, s.stream, job, n * p->blk));
@@ -1406,6 +1493,66 @@ int32_t kv_stream_wait(kv_pool_t *p, void *stream, int32_t directions)
         if (!(directions & (1 << d)) || s.issued == 0) continue;
         KV_CUDA(p, cudaStreamWaitEvent((cudaStream_t)stream, s.ev_end[s.issued % KV_SLOTS], 0));
     }
+    return KV_OK;
+}
+
+int32_t kv_completion_event(kv_pool_t *p, int32_t direction, void **event)
+{
+    if (!p || !event || (direction != 0 && direction != 1)) return KV_ERR_INVALID_ARG;
+    const DirState &s = p->dir[direction];
+    *event = s.issued ? (void *)s.ev_end[s.issued % KV_SLOTS] : nullptr;
+    return KV_OK;
+}
+
+int32_t kv_pool_set_ctas(kv_pool_t *p, int32_t ctas_out, int32_t ctas_in)
+{
+    if (!p) return KV_ERR_INVALID_ARG;
+    if (ctas_out < 0 || ctas_in < 0) return fail(p, KV_ERR_INVALID_ARG, "negative CTA count");
+    int32_t rc = kv_sync(p);
+    if (rc != KV_OK) return rc;
+    p->cfg.ctas_out = ctas_out;
+    p->cfg.ctas_in = ctas_in;
+    p->dir[0].ctas = ctas_out > 0 ? ctas_out : 64;
+    p->dir[1].ctas = ctas_in > 0 ? ctas_in : 64;
+    return KV_OK;
+}
+
+int32_t kv_debug_pair_in_bounds(int32_t src_id, int32_t dst_id, int32_t src_blocks, int32_t dst_blocks)
+{
+    return kv_pair_in_bounds(src_id, dst_id, src_blocks, dst_blocks) ? 1 : 0;
+}
+
+static int32_t check_offsets(kv_pool_t *p, const int64_t *off, int64_t n_req, int64_t n, const char *what)
+{
+    if (n_req < 0 || (n_req > 0 && !off)) return fail(p, KV_ERR_INVALID_ARG, "bad request offsets");
+    if (n_req == 0) return n == 0 ? KV_OK : fail(p, KV_ERR_INVALID_ARG, "blocks listed but no request offsets");
+    if (off[0] != 0 || off[n_req] != n) {
+        snprintf(p->err, 256, "%s request offsets must start at 0 and end at the list length", what);
+        return KV_ERR_INVALID_ARG;
+    }
+    for (int64_t k = 0; k < n_req; ++k)
+        if (off[k + 1] < off[k]) {
+            snprintf(p->err, 256, "%s request offsets must not decrease", what);
+            return KV_ERR_INVALID_ARG;
+        }
+    return KV_OK;
+}
+
+int32_t kv_rotate_req(kv_pool_t *p, const int32_t *out_gpu, const int32_t *out_host, int64_t n_out,
+                      const int64_t *out_req_offsets, int64_t n_out_req,
+                      const int32_t *in_host, const int32_t *in_gpu, int64_t n_in,
+                      const int64_t *in_req_offsets, int64_t n_in_req)
+{
+    if (!p) return KV_ERR_INVALID_ARG;
+    if (n_out < 0 || n_in < 0) return fail(p, KV_ERR_INVALID_ARG, "negative count");
+    int32_t rc = check_offsets(p, out_req_offsets, n_out_req, n_out, "swap-out");
+    if (rc != KV_OK) return rc;
+    rc = check_offsets(p, in_req_offsets, n_in_req, n_in, "swap-in");
+    if (rc != KV_OK) return rc;
+    rc = kv_rotate(p, out_gpu, out_host, n_out, in_host, in_gpu, n_in);
+    if (rc != KV_OK) return rc;
+    p->stats.requests_out += n_out_req;
+    p->stats.requests_in += n_in_req;
     return KV_OK;
 }
 
@@ -1678,6 +1825,7 @@ extern "C" int32_t kv_gather_blocks_static(const void *device_base, int32_t num_
     job.status = status;
     job.wait_polls = KV_WAIT_POLLS;
     job.wait_ns = KV_WAIT_NS;
+    job.check_ids = 0;
     job.t_first = job.t_last = nullptr;
     job.dir[1] = KvDir{};
     KvDir &kd = job.dir[0];
@@ -1685,6 +1833,8 @@ extern "C" int32_t kv_gather_blocks_static(const void *device_base, int32_t num_
     kd.dst = KvSide{(unsigned long long)dst_device, blk, seg};
     kd.pairs = pairs;
     kd.n = (int)n;
+    kd.src_blocks = (int)num_gpu_blocks;
+    kd.dst_blocks = (int)n;
     kd.ctas = clamp_ctas(job, kd, sm_count > 0 ? sm_count : 1);
     kv_copy_bulk<BULK_STAGE, BULK_NS, BULK_AHEAD><<<kd.ctas, 32, BULK_STAGE * BULK_NS, st>>>(job);
     KV_CUDA(nullptr, cudaGetLastError());

@@ -15,7 +15,7 @@
 //               through a ring of shared-memory stages guarded by mbarriers; no registers or
 //               warps are spent on the payload.  Used for HBM<->HBM gather/scatter and for
 //               HBM<->mapped host memory.
-// kv_copy_ldst  every thread moves 16-byte vectors with streaming loads/stores, all loads of a
+// kv_copy_ldst  every thread moves 16-byte (or 32-byte) vectors with streaming loads/stores, all loads of a
 //               chunk issued before its stores; each warp walks the pair list cooperatively
 //               (one coalesced load of up to 32 pairs, then shuffles).
 //
@@ -26,7 +26,14 @@
 #include <cuda_runtime.h>
 #include <stdint.h>
 
-#define KV_DEV_TIMEOUT 1u
+#define KV_DEV_TIMEOUT 1u   // a bounded wait ran out
+#define KV_DEV_BAD_ID  2u   // KvJob::check_ids: a pair named a block outside its pool; the pair was skipped
+
+// The check behind KvJob::check_ids, as a plain function of the ids and the pool sizes (host and device).
+__host__ __device__ inline bool kv_pair_in_bounds(int src_id, int dst_id, int src_blocks, int dst_blocks)
+{
+    return src_id >= 0 && src_id < src_blocks && dst_id >= 0 && dst_id < dst_blocks;
+}
 
 struct KvSide {
     unsigned long long base;
@@ -40,6 +47,7 @@ struct KvDir {
                          // nullptr = the list is short and travels with the launch (KvJob::inl)
     int n;               // pairs
     int ctas;            // CTAs assigned to this direction (0 = direction absent)
+    int src_blocks, dst_blocks;   // blocks each side holds (what KvJob::check_ids compares the ids with)
 };
 
 #define KV_INLINE_PAIRS 64   // longest pair list carried in the kernel parameters (1 KiB for both directions)
@@ -55,6 +63,9 @@ struct KvJob {
     // 200 ns apart for at most `wait_ns` nanoseconds (0 = give up right after the immediate polls)
     unsigned int wait_polls;
     unsigned long long wait_ns;
+    // non-zero: before an address is formed from a pair, its ids are compared with src_blocks / dst_blocks;
+    // a pair out of bounds sets KV_DEV_BAD_ID in the status word and none of its bytes is touched
+    int check_ids;
     // optional: device words that receive the earliest start and the latest end of the launch's CTAs
     // (%globaltimer, ns); nullptr = not wanted.  The host presets them to ~0 and 0.
     unsigned long long *t_first, *t_last;
@@ -74,6 +85,15 @@ __device__ __forceinline__ int2 kv_pair(const KvJob &job, int dsel, int i)
 struct KvCursor {
     int i, p, c;
     int2 pr;
+    bool ok;             // the current pair passed the bounds check (always true when the job does not ask for it)
+
+    __device__ __forceinline__ void load_pair(const KvJob &job, int dsel)
+    {
+        const KvDir &d = job.dir[dsel];
+        pr = kv_pair(job, dsel, i);
+        ok = !job.check_ids || kv_pair_in_bounds(pr.x, pr.y, d.src_blocks, d.dst_blocks);
+        if (!ok) atomicOr(job.status, KV_DEV_BAD_ID);
+    }
 
     __device__ __forceinline__ void seek(const KvJob &job, int dsel, long long item)
     {
@@ -83,7 +103,9 @@ struct KvCursor {
         const int r = (int)(item - (long long)i * per);
         p = r / job.cps;
         c = r - p * job.cps;
-        pr = (i < d.n) ? kv_pair(job, dsel, i) : make_int2(0, 0);
+        pr = make_int2(0, 0);
+        ok = true;
+        if (i < d.n) load_pair(job, dsel);
     }
     __device__ __forceinline__ void step(const KvJob &job, int dsel)
     {
@@ -93,7 +115,7 @@ struct KvCursor {
             if (++p == job.planes) {
                 p = 0;
                 ++i;
-                if (i < d.n) pr = kv_pair(job, dsel, i);
+                if (i < d.n) load_pair(job, dsel);
             }
         }
     }
@@ -243,9 +265,9 @@ __global__ void __launch_bounds__(32, 1) kv_copy_bulk(const __grid_constant__ Kv
         if (k < n_items) {
             const int s = (int)(k % NS);
             if (k >= NS) kv_bulk_wait_read<NS - AHEAD - 1>();
-            const uint32_t nbytes = (uint32_t)ld.bytes(job);
-            kv_mbar_expect_tx(bar0 + 8 * s, nbytes);
-            kv_bulk_load(smem0 + s * STAGE, ld.src(job, d), nbytes, bar0 + 8 * s);
+            const uint32_t nbytes = ld.ok ? (uint32_t)ld.bytes(job) : 0u;
+            kv_mbar_expect_tx(bar0 + 8 * s, nbytes);        // a skipped item arrives with no bytes to wait for
+            if (ld.ok) kv_bulk_load(smem0 + s * STAGE, ld.src(job, d), nbytes, bar0 + 8 * s);
             ld.step(job, dsel);
             ++loads_issued;
         }
@@ -257,8 +279,8 @@ __global__ void __launch_bounds__(32, 1) kv_copy_bulk(const __grid_constant__ Kv
             if (!ok) break;
             ++loads_seen;
             kv_fence_async_smem();
-            kv_bulk_store(st.dst(job, d), smem0 + s * STAGE, (uint32_t)st.bytes(job));
-            kv_bulk_commit();
+            if (st.ok) kv_bulk_store(st.dst(job, d), smem0 + s * STAGE, (uint32_t)st.bytes(job));
+            kv_bulk_commit();                               // one group per item, empty for a skipped one
             st.step(job, dsel);
         }
     }
@@ -274,10 +296,31 @@ __global__ void __launch_bounds__(32, 1) kv_copy_bulk(const __grid_constant__ Kv
 }
 
 // ------------------------------------------------------------------------------------------------
-// Load/store kernel: THREADS threads, each moving up to UNROLL 16-byte vectors per item.
-template <int THREADS, int UNROLL>
+// 32-byte vectors (sm_100: 256-bit global loads and stores).  Addresses must be 32-byte aligned.
+struct KvVec32 {
+    unsigned int w[8];
+};
+__device__ __forceinline__ KvVec32 kv_ld32(const void *p)
+{
+    KvVec32 r;
+    asm volatile("ld.global.cs.v8.b32 {%0, %1, %2, %3, %4, %5, %6, %7}, [%8];"
+                 : "=r"(r.w[0]), "=r"(r.w[1]), "=r"(r.w[2]), "=r"(r.w[3]), "=r"(r.w[4]), "=r"(r.w[5]), "=r"(r.w[6]), "=r"(r.w[7])
+                 : "l"(p)
+                 : "memory");
+    return r;
+}
+__device__ __forceinline__ void kv_st32(void *p, const KvVec32 &r)
+{
+    asm volatile("st.global.cs.v8.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8};" ::"l"(p), "r"(r.w[0]), "r"(r.w[1]), "r"(r.w[2]),
+                 "r"(r.w[3]), "r"(r.w[4]), "r"(r.w[5]), "r"(r.w[6]), "r"(r.w[7])
+                 : "memory");
+}
+
+// Load/store kernel: THREADS threads, each moving up to UNROLL vectors of VEC bytes (16 or 32) per item.
+template <int THREADS, int UNROLL, int VEC>
 __global__ void __launch_bounds__(THREADS) kv_copy_ldst(const __grid_constant__ KvJob job)
 {
+    static_assert(VEC == 16 || VEC == 32, "16- or 32-byte vectors");
     int dsel;
     long long lo, hi;
     if (!kv_my_range(job, dsel, lo, hi)) return;
@@ -300,23 +343,39 @@ __global__ void __launch_bounds__(THREADS) kv_copy_ldst(const __grid_constant__ 
         }
         const int sid = __shfl_sync(0xffffffffu, mine.x, i - win);
         const int did = __shfl_sync(0xffffffffu, mine.y, i - win);
+        const bool ok = !job.check_ids || kv_pair_in_bounds(sid, did, d.src_blocks, d.dst_blocks);
+        if (!ok && threadIdx.x == 0) atomicOr(job.status, KV_DEV_BAD_ID);
         const long long inner = (long long)c * job.chunk;
-        const uint4 *src = reinterpret_cast<const uint4 *>(d.src.base + (long long)sid * d.src.blk_stride +
-                                                          (long long)p * d.src.plane_stride + inner);
-        uint4 *dst = reinterpret_cast<uint4 *>(d.dst.base + (long long)did * d.dst.blk_stride +
-                                               (long long)p * d.dst.plane_stride + inner);
+        const unsigned char *src = reinterpret_cast<const unsigned char *>(d.src.base + (long long)sid * d.src.blk_stride +
+                                                                          (long long)p * d.src.plane_stride + inner);
+        unsigned char *dst = reinterpret_cast<unsigned char *>(d.dst.base + (long long)did * d.dst.blk_stride +
+                                                               (long long)p * d.dst.plane_stride + inner);
         const int left = job.seg - c * job.chunk;
-        const int nvec = (left < job.chunk ? left : job.chunk) >> 4;
-        uint4 v[UNROLL];
+        const int nvec = ok ? (left < job.chunk ? left : job.chunk) / VEC : 0;      // a pair out of bounds moves nothing
+        if constexpr (VEC == 16) {
+            uint4 v[UNROLL];
 #pragma unroll
-        for (int u = 0; u < UNROLL; ++u) {
-            const int q = u * THREADS + (int)threadIdx.x;
-            if (q < nvec) v[u] = __ldcs(src + q);
-        }
+            for (int u = 0; u < UNROLL; ++u) {
+                const int q = u * THREADS + (int)threadIdx.x;
+                if (q < nvec) v[u] = __ldcs(reinterpret_cast<const uint4 *>(src) + q);
+            }
 #pragma unroll
-        for (int u = 0; u < UNROLL; ++u) {
-            const int q = u * THREADS + (int)threadIdx.x;
-            if (q < nvec) __stcs(dst + q, v[u]);
+            for (int u = 0; u < UNROLL; ++u) {
+                const int q = u * THREADS + (int)threadIdx.x;
+                if (q < nvec) __stcs(reinterpret_cast<uint4 *>(dst) + q, v[u]);
+            }
+        } else {
+            KvVec32 v[UNROLL];
+#pragma unroll
+            for (int u = 0; u < UNROLL; ++u) {
+                const int q = u * THREADS + (int)threadIdx.x;
+                if (q < nvec) v[u] = kv_ld32(src + (size_t)q * 32);
+            }
+#pragma unroll
+            for (int u = 0; u < UNROLL; ++u) {
+                const int q = u * THREADS + (int)threadIdx.x;
+                if (q < nvec) kv_st32(dst + (size_t)q * 32, v[u]);
+            }
         }
         if (++c == job.cps) {
             c = 0;

@@ -15,7 +15,8 @@
         Rotation beside compute (the paper's cross-iteration pipeline, section 4.3.2, hides transfers
         behind model execution): a rotation of 2 GiB each way runs while a stand-in for a decode step
         (back-to-back element-wise kernels over 1 GiB on a third stream: HBM-bound, every SM busy) runs too.  Reports
-        how much each slows the other, for the staged and the zero-copy path.
+        how much each slows the other, for the staged path and for the zero-copy path with 8, 16, 32 and
+        64 CTAs per direction (how many SMs the rotation needs beside compute).
 
     python -m paper_2601_20309_b200.sweep latency [--out FILE]
         Call-to-completion time of small rotations (1 .. 256 blocks each way, 8B shape, scattered ids):
@@ -169,8 +170,12 @@ def overlap(out) -> None:
         return e0, e1
 
     rows = []
-    for name, pid in (("staged", B.KV_PATH_STAGED), ("zerocopy", B.KV_PATH_ZEROCOPY)):
+    # the zero-copy kernels occupy SMs for the whole transfer: how many CTAs per direction they need beside
+    # compute is the sizing question (the staged path's pack / unpack kernels run for about 1 % of the time)
+    cases = [("staged", B.KV_PATH_STAGED, 0)] + [("zerocopy", B.KV_PATH_ZEROCOPY, c) for c in (8, 16, 32, 64)]
+    for name, pid, ctas in cases:
         pool.kv_pool_set_path(pid, pid)
+        pool.kv_pool_set_ctas(ctas, ctas)
         for _ in range(2):                                     # warm-up
             pool.kv_rotate(rot.out_gpu, rot.out_host, rot.in_host, rot.in_gpu)
             pool.kv_sync()
@@ -198,7 +203,7 @@ def overlap(out) -> None:
         # the compute ran beside the rotation for rot/(k*step) of its time; scale its slowdown to that share
         r_ms, s_ms = min(both_rot), min(both_step)
         share = min(1.0, r_ms / (k * s_ms))
-        rec = {"path": name, "rotate_alone_gbs": round(nbytes / rot_alone / 1e6, 1), "rotate_beside_compute_gbs": round(nbytes / r_ms / 1e6, 1),
+        rec = {"path": name, "ctas_per_direction": ctas if ctas else None, "rotate_alone_gbs": round(nbytes / rot_alone / 1e6, 1), "rotate_beside_compute_gbs": round(nbytes / r_ms / 1e6, 1),
                "compute_alone_tbs": round(2 * (1 << 30) / step_alone / 1e9, 2), "compute_beside_rotate_tbs": round(2 * (1 << 30) / s_ms / 1e9, 2),
                "compute_slowdown_pct_over_whole_run": round(100 * (s_ms / step_alone - 1), 2),
                "compute_slowdown_pct_while_rotating": round(100 * (s_ms / step_alone - 1) / share, 2),
@@ -206,19 +211,19 @@ def overlap(out) -> None:
         rows.append(rec)
         _emit(rec, out)
     pool.destroy()
-    print("\n| path | rotate alone GB/s | rotate beside compute GB/s | compute alone TB/s | compute beside rotate TB/s | "
-          "compute slowdown while rotating | rotate slowdown |\n|---|---|---|---|---|---|---|")
+    print("\n| path | CTAs per direction | rotate alone GB/s | rotate beside compute GB/s | compute alone TB/s | compute beside rotate TB/s | "
+          "compute slowdown while rotating | rotate slowdown |\n|---|---|---|---|---|---|---|---|")
     for r in rows:
-        print(f"| {r['path']} | {r['rotate_alone_gbs']} | {r['rotate_beside_compute_gbs']} | {r['compute_alone_tbs']} | "
+        print(f"| {r['path']} | {r['ctas_per_direction'] or '-'} | {r['rotate_alone_gbs']} | {r['rotate_beside_compute_gbs']} | {r['compute_alone_tbs']} | "
               f"{r['compute_beside_rotate_tbs']} | {r['compute_slowdown_pct_while_rotating']} % | {r['rotate_slowdown_pct']} % |")
 
 
-def latency(out) -> None:
+def latency(out, block_size: int = 16) -> None:
     import time
     import numpy as np
     import torch
-    shape = W.SHAPE_8B
-    nb = 4096
+    shape = W.KVShape(32, block_size)
+    nb = 4096 * 16 // block_size if block_size < 16 else 4096
     dev = torch.empty(nb * shape.block_bytes, dtype=torch.uint8, device="cuda:0")
     pool = B.KVPool(shape.num_layers, shape.block_size, shape.kv_heads, shape.head_dim, nb, nb, dev.data_ptr())
     rng = np.random.default_rng(3)
@@ -300,6 +305,7 @@ def main() -> None:
     ap.add_argument("--out", default=None)
     ap.add_argument("--max-payload-gb", type=float, default=4.0)
     ap.add_argument("--b-xfer", type=int, default=2400, help="budget: blocks per step, both directions together")
+    ap.add_argument("--block-size", type=int, default=16, help="latency: tokens per block (8 = 1 MiB blocks, 16 = 2 MiB, 32 = 4 MiB)")
     ap.add_argument("--device-layout", choices=["layer-first", "block-first"], default="layer-first",
                     help="paths: device pool layout (block-first = the paper's redesigned storage order)")
     a = ap.parse_args()
@@ -314,7 +320,7 @@ def main() -> None:
     elif a.what == "overlap":
         overlap(out)
     elif a.what == "latency":
-        latency(out)
+        latency(out, a.block_size)
     else:
         budget(out, a.b_xfer)
 

@@ -43,6 +43,15 @@ def test_shape_helpers_need_no_device():
 def test_struct_sizes_match_the_header_layout():
     # natural alignment on both sides; a mismatch here means the ctypes mirror drifted from the header
     assert C.sizeof(B.kv_pool_config_t) == 112
-    assert C.sizeof(B.kv_stats_t) == 128
+    assert C.sizeof(B.kv_stats_t) == 144
     assert C.sizeof(B.kv_link_probe_t) == 56
     assert C.sizeof(B.kv_probe_spec_t) == 56
+
+
+def test_bounds_predicate_of_the_debug_flag():
+    """What the kernels check under KV_FLAG_DEBUG_BOUNDS, as the plain host function it is written as."""
+    ok = B.kv_debug_pair_in_bounds
+    assert ok(0, 0, 1, 1) and ok(27, 511, 28, 512)
+    assert not ok(28, 0, 28, 512) and not ok(0, 512, 28, 512)       # one past the end, either side
+    assert not ok(-1, 0, 28, 512) and not ok(0, -1, 28, 512)        # negative ids
+    assert not ok(0, 0, 0, 5) and not ok(2 ** 31 - 1, 0, 2 ** 31 - 1, 1)

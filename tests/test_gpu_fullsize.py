@@ -172,12 +172,14 @@ def test_config5_full_shape_replay_2000_steps():
         t.close()
 
 
-@pytest.mark.parametrize("bs,contiguous,payload", [(8, False, 2e9), (64, True, 4e9), (32, False, 4e9)],
-                         ids=["block8-random-2GB", "block64-contiguous-4GB", "block32-random-4GB"])
+@pytest.mark.parametrize("bs,contiguous,payload", [(8, False, 2e9), (64, True, 4e9), (32, False, 4e9), (16, False, 8 << 30)],
+                         ids=["block8-random-2GB", "block64-contiguous-4GB", "block32-random-4GB", "block16-random-8GiB"])
 def test_config4_sweep_cells_at_full_payload(bs, contiguous, payload):
     """Cells of the block-size / fragmentation sweep at full payload, default path: 1 MiB blocks with random
     tables (the zero-copy kernels), 8 MiB blocks with contiguous tables (long merged transfers), 4 MiB
-    blocks with random tables (uniform two-block transfers).  Each direction alone, then both at once."""
+    blocks with random tables (uniform two-block transfers), and the cell of the paper's bandwidth table
+    (section 5.3.3): 2 MiB blocks, random tables, 8 GiB = 32768 tokens of 256 KB each way.  Each direction
+    alone, then both at once."""
     w = W.config4_sweep_case(bs, contiguous, payload)
     t = _FullSize(w)
     try:

@@ -467,10 +467,13 @@ def test_caller_supplied_host_memory_is_page_locked_and_stays_inside_its_bounds(
     dict(path=1, path_in=2), dict(path=2, path_in=1), dict(path=3, path_in=1), dict(path=3, ce_streams=4),
     dict(path=4, ce_streams=2), dict(path=1, ctas_out=3, ctas_in=148), dict(path=1, flags=4, ctas_out=5, ctas_in=9),
     dict(path=2, staging_bytes=1), dict(path=0, flags=8),
+    dict(path=1, link_variant=1), dict(path=1, link_variant=2), dict(path=1, flags=2, link_variant=1),
+    dict(path=1, flags=4, link_variant=2, ctas_out=7, ctas_in=7),
 ], ids=lambda k: "-".join(f"{a}{b}" for a, b in k.items()))
 def test_tuning_knobs_do_not_change_results(knobs):
     """A different path per direction, several copy-engine streams, odd CTA counts, the smallest staging,
-    kernel timing: every setting must give the oracle's bytes."""
+    kernel timing, the other shapes of the zero-copy kernels' transfers (32 and 64 KiB bulk copies, 32-byte
+    vectors): every setting must give the oracle's bytes."""
     w = W.config2_8b(nb_gpu=320, nb_host=448, n_req=16, median=96, max_tokens=512, n_rot=4)
     p = _pair(w.shape, w.nb_gpu, w.nb_host, seed=w.seed, **knobs)
     try:
