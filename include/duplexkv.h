@@ -212,25 +212,30 @@ int32_t kv_rotate_req(kv_pool_t *pool,
                       const int64_t *in_req_offsets, int64_t n_in_req);
 
 /*
- * What copy-engine transfers the STAGED path would make for one direction of a call (no pool, no GPU):
- * the list is sorted by host id; where the ids form long runs (8 blocks and more on average) each run
- * is one transfer and equal runs at a constant spacing share one strided transfer; otherwise every
- * transfer carries exactly two blocks (neighbours in the sorted list, any distance apart in host
- * memory), because transfers of one size keep the two copy engines of a rotation in step (section
- * 4.3.2's "merge small segments into large transfers", bounded here by what the ids allow).  The sequence
- * is cut into chunks of at most half_blocks blocks (one staging half each; about four chunks for a
- * call that would fit one half).
+ * What copy-engine transfers the STAGED path would make for one direction of a call (no pool, no GPU).
+ * Where the host ids form long runs (8 blocks and more on average) the list is taken in ascending order
+ * of host id, each run is one transfer and equal runs at a constant spacing share one strided transfer.
+ * Otherwise every block counts as a single: four blocks whose ids form a 2 x 2 lattice (a, a+g, a+kg,
+ * a+kg+g) share one 3-D transfer, the blocks left over travel two per transfer (neighbours in ascending
+ * order, any distance apart in host memory), lattices first -- transfers of few sizes keep the two copy
+ * engines of a rotation in step (section 4.3.2's "merge small segments into large transfers", bounded
+ * here by what the ids allow).  The sequence is cut into chunks of at most half_blocks blocks (one
+ * staging half each; about four chunks for a call that would fit one half, a single chunk for a call of
+ * 128 MiB or less).
  *   host_ids   HOST array of n host block ids (direction 0: swap-out destinations, 1: swap-in sources)
  *   ops        HOST array of ops_cap entries, filled in issue order; *n_ops = transfers needed
  *              (with ops_cap == 0 only the count is returned)
  *   order      HOST array of n entries or NULL: order[k] = index in host_ids of the block that takes
- *              staging position k (= position k of the sorted list)
- * A transfer moves rows x blocks_per_row blocks: row r covers host blocks host_block + r*pitch_blocks ..
- * + blocks_per_row - 1 and staging positions first_position + r*blocks_per_row .. of the sorted list.
+ *              staging position k (the staging order: the blocks of each transfer side by side, transfers
+ *              in issue order)
+ * A transfer moves slices x rows x blocks_per_row blocks: row r of slice s covers host blocks
+ * host_block + s*slice_pitch_blocks + r*pitch_blocks .. + blocks_per_row - 1, and the transfer's blocks
+ * take staging positions first_position .. in (slice, row, block) order.
  */
 typedef struct {
     int64_t host_block, first_position, pitch_blocks;
-    int32_t rows, blocks_per_row, chunk, pad_;
+    int32_t rows, blocks_per_row, chunk, slices;
+    int64_t slice_pitch_blocks;
 } kv_plan_op_t;
 int32_t kv_plan_staged(int64_t blk_bytes, int64_t half_blocks, int32_t direction, const int32_t *host_ids, int64_t n,
                        kv_plan_op_t *ops, int64_t ops_cap, int64_t *n_ops, int32_t *order);
@@ -345,6 +350,9 @@ int32_t kv_probe_link(int32_t device_id, int64_t bytes, int32_t reps, kv_link_pr
  * total_bytes/copy_bytes copy-engine transfers of copy_bytes back to back on one stream per direction.
  * rows <= 1: plain transfers.  rows > 1: strided 2-D transfers of `rows` rows of copy_bytes/rows bytes,
  * row r at start + r*host_pitch on the host and start + r*dev_pitch on the device (0 = rows packed).
+ * slices > 1 (with rows > 1): 3-D transfers of `slices` x `rows` rows; on the host slice s starts
+ * s*host_slice_rows*host_pitch after the first (host_slice_rows >= rows), on the device rows and slices are
+ * packed at dev_pitch.  That is how four blocks on a 2 x 2 lattice of host addresses travel in one transfer.
  * The transfers start at consecutive places of span_bytes-sized buffers (wrapping), or at seeded
  * pseudo-random row-aligned offsets when scattered != 0.  One warm-up round, then `rounds` timed
  * ones; the best is kept.  out->bytes = copy_bytes, out->reps = transfers per round.
@@ -353,6 +361,7 @@ typedef struct {
     int64_t copy_bytes, total_bytes, span_bytes;
     int32_t scattered, rounds;
     int64_t rows, host_pitch, dev_pitch;
+    int64_t slices, host_slice_rows;
 } kv_probe_spec_t;
 int32_t kv_probe_link_ex(int32_t device_id, const kv_probe_spec_t *spec, kv_link_probe_t *out);
 

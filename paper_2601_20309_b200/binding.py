@@ -74,7 +74,8 @@ class kv_link_probe_t(C.Structure):
 class kv_probe_spec_t(C.Structure):
     _fields_ = [("copy_bytes", C.c_int64), ("total_bytes", C.c_int64), ("span_bytes", C.c_int64),
                 ("scattered", C.c_int32), ("rounds", C.c_int32),
-                ("rows", C.c_int64), ("host_pitch", C.c_int64), ("dev_pitch", C.c_int64)]
+                ("rows", C.c_int64), ("host_pitch", C.c_int64), ("dev_pitch", C.c_int64),
+                ("slices", C.c_int64), ("host_slice_rows", C.c_int64)]
 
 
 class kv_pool_shape_t(C.Structure):
@@ -97,7 +98,8 @@ class kv_table_stats_t(C.Structure):
 
 class kv_plan_op_t(C.Structure):
     _fields_ = [("host_block", C.c_int64), ("first_position", C.c_int64), ("pitch_blocks", C.c_int64),
-                ("rows", C.c_int32), ("blocks_per_row", C.c_int32), ("chunk", C.c_int32), ("pad_", C.c_int32)]
+                ("rows", C.c_int32), ("blocks_per_row", C.c_int32), ("chunk", C.c_int32), ("slices", C.c_int32),
+                ("slice_pitch_blocks", C.c_int64)]
 
 
 EXPORTS = ["kv_pool_create", "kv_pool_destroy", "kv_pool_set_path", "kv_swap_out", "kv_swap_in", "kv_rotate", "kv_sync",
@@ -250,8 +252,9 @@ def kv_probe_link(device_id: int = 0, nbytes: int = 256 << 20, reps: int = 4) ->
 
 def kv_probe_link_ex(device_id: int, copy_bytes: int, total_bytes: int, span_bytes: int,
                      scattered: bool = False, rounds: int = 3, rows: int = 1, host_pitch: int = 0,
-                     dev_pitch: int = 0) -> dict:
-    spec = kv_probe_spec_t(copy_bytes, total_bytes, span_bytes, int(scattered), rounds, rows, host_pitch, dev_pitch)
+                     dev_pitch: int = 0, slices: int = 1, host_slice_rows: int = 0) -> dict:
+    spec = kv_probe_spec_t(copy_bytes, total_bytes, span_bytes, int(scattered), rounds, rows, host_pitch, dev_pitch,
+                           slices, host_slice_rows)
     out = kv_link_probe_t()
     rc = lib().kv_probe_link_ex(device_id, C.byref(spec), C.byref(out))
     if rc != KV_OK:

@@ -30,6 +30,12 @@
         device time of every step's rotation, against the 70 ms a model step takes in the paper
         (section 5.3.4), i.e. how often the transfer would not hide behind the step.
 
+    python -m paper_2601_20309_b200.sweep handoff [--out FILE]
+        What a hand-off between the copy engine and a kernel costs while the host link is busy (plain torch
+        streams, no library call): a host-to-device copy followed by a tiny kernel that waits for it, and a
+        tiny kernel followed by a device-to-host copy that waits for it, on one stream or across two, with
+        the other direction idle or saturated.  This is the price of every chunk boundary of the staged path.
+
 All print one JSON object per line and, at the end, a markdown table.
 """
 from __future__ import annotations
@@ -71,6 +77,11 @@ def probe(out) -> None:
         ("2 rows x 4 MiB, host pitch 64 MiB", dict(copy_bytes=8 * M, rows=2, host_pitch=64 * M)),
         ("4 rows x 2 MiB, host pitch 64 MiB", dict(copy_bytes=8 * M, rows=4, host_pitch=64 * M)),
         ("8 rows x 2 MiB, host pitch 64 MiB", dict(copy_bytes=16 * M, rows=8, host_pitch=64 * M)),
+        # four blocks whose host addresses form a 2 x 2 lattice (a, a+g, a+kg, a+kg+g) as one 3-D transfer
+        ("2 slices x 2 rows x 2 MiB (3-D), row pitch 64 MiB, slices 448 MiB apart",
+         dict(copy_bytes=8 * M, rows=2, host_pitch=64 * M, slices=2, host_slice_rows=7)),
+        ("2 slices x 2 rows x 1 MiB (3-D), row pitch 64 MiB, slices 448 MiB apart",
+         dict(copy_bytes=4 * M, rows=2, host_pitch=64 * M, slices=2, host_slice_rows=7)),
     ]
     for name, kw in shapes:
         total = G if kw["copy_bytes"] >= 256 * K else G // 4
@@ -265,6 +276,79 @@ def latency(out, block_size: int = 16) -> None:
               f"{r['zerocopy_us']} | {r['ce2d_us']} | {r['auto_over_best_pct']} % | {r['auto_untimed_us']} | {r['link_floor_us']} |")
 
 
+def handoff(out) -> None:
+    import torch
+    dev = "cuda:0"
+    hsrc = torch.empty(256 * M, dtype=torch.uint8).pin_memory()
+    hdst = torch.empty(1024 * M, dtype=torch.uint8).pin_memory()
+    dsrc = torch.empty(1024 * M, dtype=torch.uint8, device=dev)
+    ddst = torch.empty(256 * M, dtype=torch.uint8, device=dev)
+    small = torch.zeros(1024, device=dev)
+    s_a, s_b, s_k = torch.cuda.Stream(), torch.cuda.Stream(), torch.cuda.Stream()
+
+    def median_of(fn, reps=7):
+        res = sorted((fn() for _ in range(reps)), key=lambda r: r[1])
+        return res[len(res) // 2]
+
+    def copy_then_kernel(size_mib, busy, same_stream):
+        torch.cuda.synchronize()
+        e0, e1, e2 = (torch.cuda.Event(enable_timing=True) for _ in range(3))
+        if busy:
+            with torch.cuda.stream(s_b):
+                hdst.copy_(dsrc, non_blocking=True)                # 1 GiB device to host: outlasts everything below
+        with torch.cuda.stream(s_a):
+            e0.record()
+            ddst[:size_mib * M].copy_(hsrc[:size_mib * M], non_blocking=True)
+            e1.record()
+            if same_stream:
+                small.add_(1)
+                e2.record()
+        if not same_stream:
+            s_k.wait_event(e1)
+            with torch.cuda.stream(s_k):
+                small.add_(1)
+                e2.record()
+        torch.cuda.synchronize()
+        return e0.elapsed_time(e1), e1.elapsed_time(e2)
+
+    def kernel_then_copy(size_mib, busy, same_stream):
+        torch.cuda.synchronize()
+        e0, e1, e2 = (torch.cuda.Event(enable_timing=True) for _ in range(3))
+        if busy:
+            with torch.cuda.stream(s_b):
+                for _ in range(4):
+                    ddst.copy_(hsrc, non_blocking=True)            # 1 GiB host to device in all
+        with torch.cuda.stream(s_a if same_stream else s_k):
+            e0.record()
+            small.add_(1)
+            e1.record()
+        if not same_stream:
+            s_a.wait_event(e1)
+        with torch.cuda.stream(s_a):
+            hdst[:size_mib * M].copy_(dsrc[:size_mib * M], non_blocking=True)
+            e2.record()
+        torch.cuda.synchronize()
+        return e0.elapsed_time(e1), e1.elapsed_time(e2)
+
+    rows = []
+    for size in (16, 64):
+        for busy in (False, True):
+            for same in (False, True):
+                c, h = median_of(lambda: copy_then_kernel(size, busy, same))
+                k, t = median_of(lambda: kernel_then_copy(size, busy, same))
+                rate = (55.5e9 if not busy else 49.5e9), (57.2e9 if not busy else 49.5e9)
+                rec = {"copy_mib": size, "other_direction_busy": busy, "same_stream": same,
+                       "h2d_copy_ms": round(c, 3), "h2d_copy_end_to_kernel_end_us": round(h * 1e3, 1),
+                       "kernel_end_to_d2h_copy_end_ms": round(t, 3),
+                       "of_which_before_the_copy_starts_us": round((t - size * M / rate[1] * 1e3) * 1e3, 1)}
+                rows.append(rec)
+                _emit(rec, out)
+    print("\n| copy MiB | other direction | streams | H2D copy ms | copy end to kernel end us | kernel end to D2H copy end ms | of which before the copy starts, us (copy at the probe's rate) |\n|---|---|---|---|---|---|---|")
+    for r in rows:
+        print(f"| {r['copy_mib']} | {'saturated' if r['other_direction_busy'] else 'idle'} | {'one' if r['same_stream'] else 'two'} | {r['h2d_copy_ms']} | "
+              f"{r['h2d_copy_end_to_kernel_end_us']} | {r['kernel_end_to_d2h_copy_end_ms']} | {r['of_which_before_the_copy_starts_us']} |")
+
+
 def budget(out, b_xfer: int) -> None:
     import numpy as np
     import torch
@@ -301,7 +385,7 @@ def budget(out, b_xfer: int) -> None:
 
 def main() -> None:
     ap = argparse.ArgumentParser()
-    ap.add_argument("what", choices=["probe", "paths", "overlap", "latency", "budget"])
+    ap.add_argument("what", choices=["probe", "paths", "overlap", "latency", "budget", "handoff"])
     ap.add_argument("--out", default=None)
     ap.add_argument("--max-payload-gb", type=float, default=4.0)
     ap.add_argument("--b-xfer", type=int, default=2400, help="budget: blocks per step, both directions together")
@@ -321,6 +405,8 @@ def main() -> None:
         overlap(out)
     elif a.what == "latency":
         latency(out, a.block_size)
+    elif a.what == "handoff":
+        handoff(out)
     else:
         budget(out, a.b_xfer)
 

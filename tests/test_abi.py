@@ -45,7 +45,7 @@ def test_struct_sizes_match_the_header_layout():
     assert C.sizeof(B.kv_pool_config_t) == 112
     assert C.sizeof(B.kv_stats_t) == 144
     assert C.sizeof(B.kv_link_probe_t) == 56
-    assert C.sizeof(B.kv_probe_spec_t) == 56
+    assert C.sizeof(B.kv_probe_spec_t) == 72
 
 
 def test_bounds_predicate_of_the_debug_flag():

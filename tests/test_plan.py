@@ -14,51 +14,88 @@ def check_plan(host_ids, half_blocks, direction, blk=BLK):
     ops, order = B.kv_plan_staged(blk, half_blocks, direction, host_ids)
     n = len(host_ids)
     assert sorted(order.tolist()) == list(range(n))                         # a permutation of the list
-    sorted_ids = host_ids[order]
-    assert np.all(np.diff(sorted_ids) >= 0)                                 # staging order = ascending host id
+    staged_ids = host_ids[order]                                            # host id at every staging position
     pos = 0
     per_chunk = {}
     for op in ops:
-        assert op["first_position"] == pos                                  # issue order walks the sorted list
-        assert op["rows"] >= 1 and op["blocks_per_row"] >= 1
-        for r in range(op["rows"]):
-            for j in range(op["blocks_per_row"]):
-                want = op["host_block"] + r * op["pitch_blocks"] + j
-                assert sorted_ids[pos] == want, (op, r, j)
-                pos += 1
+        assert op["first_position"] == pos                                  # issue order walks the staging order
+        assert op["rows"] >= 1 and op["blocks_per_row"] >= 1 and op["slices"] >= 1
+        for s in range(op["slices"]):
+            for r in range(op["rows"]):
+                for j in range(op["blocks_per_row"]):
+                    want = op["host_block"] + s * op["slice_pitch_blocks"] + r * op["pitch_blocks"] + j
+                    assert staged_ids[pos] == want, (op, s, r, j)
+                    pos += 1
         if op["rows"] > 1:
             assert op["pitch_blocks"] >= op["blocks_per_row"]                # rows do not overlap in host memory
             assert op["pitch_blocks"] * blk <= 2 ** 31 - 1                   # what a strided transfer accepts
-        per_chunk[op["chunk"]] = per_chunk.get(op["chunk"], 0) + op["rows"] * op["blocks_per_row"]
+        if op["slices"] > 1:
+            assert op["rows"] > 1 and op["slice_pitch_blocks"] % op["pitch_blocks"] == 0      # a whole number of row pitches
+            assert op["slice_pitch_blocks"] >= op["rows"] * op["pitch_blocks"]                # slices do not interleave
+        per_chunk[op["chunk"]] = per_chunk.get(op["chunk"], 0) + op["slices"] * op["rows"] * op["blocks_per_row"]
     assert pos == n                                                          # every block exactly once
     assert sorted(per_chunk) == list(range(len(per_chunk)))                  # chunks numbered in order
     assert all(v <= half_blocks for v in per_chunk.values())                 # a chunk fits a staging half
+    if all(op["slices"] == 1 for op in ops):
+        assert np.all(np.diff(staged_ids) >= 0)                             # without lattices: ascending host id
     return ops, per_chunk
+
+
+def _blocks(op):
+    return op["slices"] * op["rows"] * op["blocks_per_row"]
 
 
 @pytest.mark.parametrize("direction", [0, 1])
 @pytest.mark.parametrize("seed", range(5))
-def test_scattered_ids_travel_two_per_transfer_all_alike(seed, direction):
+def test_scattered_ids_travel_four_or_two_per_transfer(seed, direction):
     rng = np.random.default_rng(seed)
     n = int(rng.integers(50, 700))
     ids = rng.choice(60_000, n, replace=False)
     ops, chunks = check_plan(ids, 512, direction)
-    sizes = [op["rows"] * op["blocks_per_row"] for op in ops]
-    # ids more than 2 GiB apart cannot share a strided transfer; everything else is a pair
-    assert sizes.count(2) >= len(sizes) - 1 - sum(1 for a, b in zip(np.sort(ids), np.sort(ids)[1:]) if (b - a) * BLK > 2 ** 31 - 1)
-    assert max(sizes) == 2
+    sizes = [_blocks(op) for op in ops]
+    # lattices of four first, then pairs; ids more than 2 GiB apart cannot share a strided transfer
+    far = sum(1 for a, b in zip(np.sort(ids), np.sort(ids)[1:]) if (b - a) * BLK > 2 ** 31 - 1)
+    assert set(sizes) <= {4, 2, 1} and sizes.count(1) <= 1 + far
+    assert sizes == sorted(sizes, reverse=True) or far                     # four-block transfers are issued first
+    assert all(op["slices"] == 2 and op["rows"] == 2 for op in ops if _blocks(op) == 4)
     assert len(ops) <= (n + 1) // 2 + 8
+
+
+def test_lattices_cover_most_of_a_scattered_list():
+    """1844 ids drawn from 57 220 (the density of the 8B-shaped rotation): about three quarters of the
+    blocks find a place in a four-block lattice; a denser list does better."""
+    rng = np.random.default_rng(11)
+    for n, nb, least in ((1844, 57_220, 0.65), (4096, 57_220, 0.85)):
+        ids = rng.choice(nb, n, replace=False)
+        ops, _ = check_plan(ids, 512, 0)
+        in_fours = sum(4 for op in ops if _blocks(op) == 4)
+        assert in_fours >= least * n, (n, in_fours)
+        assert all(op["pitch_blocks"] <= 256 for op in ops if _blocks(op) == 4)
+
+
+def test_hand_made_lattice():
+    # 10, 13 and 31, 34: gap 3, starts congruent modulo 3 (31 - 10 = 7 * 3): one transfer; the rest go in pairs
+    ops, _ = check_plan([34, 500, 10, 900, 31, 13, 77, 70], 64, 0)
+    four = [op for op in ops if _blocks(op) == 4]
+    assert len(four) == 1
+    assert (four[0]["host_block"], four[0]["pitch_blocks"], four[0]["slice_pitch_blocks"]) == (10, 3, 21)
+    assert [_blocks(op) for op in ops] == [4, 2, 2]
 
 
 def test_long_runs_are_merged_and_cut_at_chunk_size():
     ids = np.concatenate([np.arange(1000, 1300), np.arange(5000, 5200), np.arange(9000, 9040)])    # runs of 300, 200, 40
     rng = np.random.default_rng(0)
     ops, chunks = check_plan(rng.permutation(ids), 128, 1)
-    assert all(op["rows"] * op["blocks_per_row"] <= 128 for op in ops)
+    assert all(_blocks(op) <= 128 for op in ops)
     assert len(ops) <= 8                                                     # 300 -> 3, 200 -> 2, 40 -> 1 (or merged rows)
     assert sum(chunks.values()) == 540
-    one, _ = check_plan(np.arange(77, 77 + 64), 512, 0)                      # a call that fits one half: about four chunks
-    assert 3 <= len({op["chunk"] for op in one}) <= 6
+    one, _ = check_plan(np.arange(77, 77 + 64), 512, 0)                      # 128 MiB or less: one chunk, one transfer
+    assert len(one) == 1 and one[0]["blocks_per_row"] == 64
+    four, _ = check_plan(np.arange(77, 77 + 200), 512, 0)                    # larger, but fits one half: about four chunks,
+    sizes = [_blocks(op) for op in four]                                     # the first of a swap-out half as long
+    assert 3 <= len({op["chunk"] for op in four}) <= 6 and sizes[0] == 25 and sizes[1] == 50
+    four_in, _ = check_plan(np.arange(77, 77 + 200), 512, 1)
+    assert [_blocks(op) for op in four_in] == [50, 50, 50, 50]
 
 
 def test_short_runs_are_not_merged_into_uneven_transfers():
@@ -70,8 +107,8 @@ def test_short_runs_are_not_merged_into_uneven_transfers():
         ids += list(range(at, at + L))
         at += L + int(rng.integers(2, 50))
     ops, _ = check_plan(rng.permutation(np.array(ids[:400])), 512, 0)
-    assert {op["rows"] * op["blocks_per_row"] for op in ops} == {2}
-    assert len(ops) == 200
+    assert {_blocks(op) for op in ops} <= {4, 2}
+    assert 100 <= len(ops) <= 200
 
 
 def test_equal_runs_at_a_constant_spacing_share_one_strided_transfer():
