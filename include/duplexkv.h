@@ -58,10 +58,10 @@ extern "C" {
 #define KV_DEV_BLOCK_FIRST    1     /* [block][layer][K|V]...: the paper's redesigned storage order      */
 
 /* transfer paths (how the host link is driven) */
-#define KV_PATH_AUTO          0     /* per call.  Calls bound by fixed costs, 32 MiB or less per direction:
-                                       CE2D (blocks under 2 MiB: CE2D up to 8 MiB, ZEROCOPY above).  Larger
-                                       calls: STAGED when the copy-engine transfers the call needs would
-                                       average 3 MiB or more, else ZEROCOPY (see kv_path_for)            */
+#define KV_PATH_AUTO          0     /* per call.  8 MiB or less per direction (2 MiB for blocks under 2 MiB):
+                                       CE2D, the lowest fixed cost.  Larger calls: STAGED when the
+                                       copy-engine transfers the call needs would average 3 MiB or more,
+                                       else ZEROCOPY (see kv_path_for)                                   */
 #define KV_PATH_ZEROCOPY      1     /* SM kernels read/write mapped pinned host memory directly          */
 #define KV_PATH_STAGED        2     /* pack kernel -> contiguous HBM staging -> copy engine (and reverse)*/
 #define KV_PATH_CE2D          3     /* one strided 2-D copy-engine transfer per block, no kernel         */
@@ -330,9 +330,10 @@ const char *kv_last_error(kv_pool_t *pool);
 int64_t kv_seg_bytes(int32_t block_size, int32_t kv_heads, int32_t head_dim);
 int64_t kv_blk_bytes(int32_t num_layers, int32_t block_size, int32_t kv_heads, int32_t head_dim);
 
-/* The path KV_PATH_AUTO resolves to for blocks of blk_bytes (= kv_blk_bytes of the shape) whose host ids
- * have no neighbours in the list (such blocks travel two per transfer).  Lists with neighbouring host
- * ids make larger transfers and can go STAGED at smaller block sizes; AUTO decides that per call. */
+/* The path KV_PATH_AUTO resolves to for a large call of blocks of blk_bytes (= kv_blk_bytes of the shape) in
+ * the worst case for the copy engines: host ids with no neighbours and no lattices in the list, so that
+ * the blocks travel two per transfer.  Lists whose ids form runs or lattices make larger transfers and
+ * go STAGED at smaller block sizes too; AUTO decides that per call from the transfers it plans. */
 int32_t kv_path_for(int64_t blk_bytes);
 
 /*

@@ -22,16 +22,15 @@ namespace {
 constexpr int KV_SLOTS = 8;            // descriptor / event ring depth per direction
 constexpr int KV_MAX_CE_STREAMS = 4;
 constexpr int64_t KV_AUTO_MIN_TRANSFER = 3ll << 20;   // AUTO: staged when its transfers average 3 MiB or more
-// AUTO, calls bound by fixed costs rather than by the link (measured on 2 MiB blocks, scattered ids, call to
-// completion, two runs): one copy-engine transfer per block is the quickest or within 1.5 % of it up to 16
-// blocks each way (64 / 109 / 216 / 420-470 / 826-858 us for 1 / 2 / 4 / 8 / 16 blocks against 86 / 142 /
-// 247 / 455 / 882-900 us for the zero-copy kernels and 93 / 145 / 239 / 494 / 849-860 us staged); from 32
-// blocks on the staged pipeline is ahead and the transfer-size rule decides.  One transfer per block needs
-// blocks of 2 MiB or more to reach the kernels' rate; smaller blocks take that path only up to 8 MiB and the
-// zero-copy kernels above that.
-constexpr int64_t KV_AUTO_TINY_BYTES = 32ll << 20;
-constexpr int64_t KV_AUTO_TINY_BYTES_SMALL_BLOCKS = 8ll << 20;
-constexpr int64_t KV_AUTO_SMALL_BYTES = 32ll << 20;
+// AUTO, calls bound by fixed costs rather than by the link (measured on scattered ids, call to completion):
+// one copy-engine transfer per block is the quickest up to 8 MiB per direction of 2 MiB blocks (65 / 111 /
+// 212 us for 1 / 2 / 4 blocks each way against 85 / 141 / 231 us staged and 87 / 143 / 247 us for the
+// zero-copy kernels); from 16 MiB on the staged path (one chunk, ids in the launch parameters, four-block
+// lattices) is ahead (406 / 789 us at 8 / 16 blocks against 451 / 847 and 463 / 908) and the transfer-size
+// rule decides.  With 1 MiB blocks one transfer per block wins only up to 2 MiB (44 / 75 us for 1 / 2
+// blocks); above that the transfer-size rule picks the zero-copy kernels, which lead up to ~128 MiB.
+constexpr int64_t KV_AUTO_TINY_BYTES = 8ll << 20;
+constexpr int64_t KV_AUTO_TINY_BYTES_SMALL_BLOCKS = 2ll << 20;
 constexpr int64_t KV_MERGE_MIN_MEAN_RUN = 8;
 constexpr int64_t KV_QUAD_MAX_GAP = 256;              // STAGED, scattered ids: largest row gap (blocks) of a four-block lattice
 constexpr int KV_QUAD_PARTNERS = 6;                   //         partners tried per block when looking for lattices
@@ -570,7 +569,14 @@ void plan_transfers(const PlanParams &pp, int d, const int32_t *host_ids, int64_
         // long as the rest: its first transfer starts sooner.
         const int64_t min_chunk = std::max<int64_t>(1, (8ll << 20) / pp.blk);
         const bool one_chunk = n * pp.blk <= KV_PLAN_ONE_CHUNK_BYTES;
-        const int64_t chunk = std::min(pp.half_blocks, one_chunk ? n : std::max(min_chunk, (n + KV_PLAN_CHUNKS - 1) / KV_PLAN_CHUNKS));
+        int64_t chunk = std::min(pp.half_blocks, one_chunk ? n : std::max(min_chunk, (n + KV_PLAN_CHUNKS - 1) / KV_PLAN_CHUNKS));
+        {
+            // as many chunks as that size needs, but of equal size (a multiple of four blocks where the half
+            // allows it), so that no call ends on a chunk of a few blocks and a hand-off of its own
+            const int64_t pieces = (n + chunk - 1) / chunk;
+            const int64_t even = (((n + pieces - 1) / pieces) + 3) & ~(int64_t)3;
+            chunk = std::min(pp.half_blocks, std::max(chunk, even));
+        }
         const int64_t first = (d == 0 && n > chunk && !one_chunk) ? std::max<int64_t>(1, chunk / 2) : chunk;
         if (pp.layer_first) {
             // one strided transfer per block: `planes` rows of SEG bytes, a whole host plane apart
@@ -940,13 +946,12 @@ int32_t run_calls(kv_pool *p, DirCall *calls, int ncalls, const bool *wait_other
             const DirState &o = p->dir[1 - calls[k].d];
             wait_ev[k] = o.ev_end[o.issued % KV_SLOTS];
         }
-    // KV_PATH_AUTO is settled per call.  A call that moves little is bound by its fixed costs, not by the
-    // link: up to KV_AUTO_TINY_BYTES per direction (less for blocks under 2 MiB) it goes as one copy-engine
-    // transfer per block, up to KV_AUTO_SMALL_BYTES to the zero-copy kernels (one launch, no staging pipeline).  Otherwise the staged
-    // transfers are planned first (cheap: a sort of the ids) and the staged path is taken when its transfers
-    // would carry KV_AUTO_MIN_TRANSFER bytes or more on average, the zero-copy kernels when not.  Both
-    // directions of a rotate take the same path (a kernel on one direction starves the copy engine on the
-    // other).
+    // KV_PATH_AUTO is settled per call.  A call that moves very little (KV_AUTO_TINY_BYTES per direction, less
+    // for blocks under 2 MiB) is all fixed cost and goes as one copy-engine transfer per block.  Otherwise the
+    // staged transfers are planned first (cheap: a sort of the ids and one sweep over them) and the staged
+    // path is taken when its transfers would carry KV_AUTO_MIN_TRANSFER bytes or more on average, the
+    // zero-copy kernels when not.  Both directions of a rotate take the same path (a kernel on one direction
+    // starves the copy engine on the other).
     {
         int64_t largest = 0;
         for (int k = 0; k < ncalls; ++k) {
@@ -956,8 +961,6 @@ int32_t run_calls(kv_pool *p, DirCall *calls, int ncalls, const bool *wait_other
         int chosen;
         if (largest <= (p->blk >= (2ll << 20) ? KV_AUTO_TINY_BYTES : KV_AUTO_TINY_BYTES_SMALL_BLOCKS)) {
             chosen = KV_PATH_CE2D;
-        } else if (largest <= KV_AUTO_SMALL_BYTES) {
-            chosen = KV_PATH_ZEROCOPY;
         } else {
             int64_t bytes = 0, ops = 0;
             for (int k = 0; k < ncalls; ++k) {
@@ -1090,9 +1093,9 @@ int32_t kv_path_for(int64_t blk_bytes)
     // Measured on B200 behind PCIe Gen5 x16, both directions busy: a copy-engine transfer costs a fixed
     // start-up (about 10 us with the other direction busy) plus its bytes, so the staged path wins once its
     // transfers carry 3 MiB or more; below that the zero-copy kernels, which pay no per-transfer cost,
-    // are ahead.  Blocks with no neighbours in host memory travel two per transfer, hence this rule for
-    // fully scattered ids; a pool on KV_PATH_AUTO applies the same threshold to the transfers each call
-    // actually needs, so lists with neighbouring host ids go staged at any block size.
+    // are ahead.  Blocks with no neighbours in host memory travel at least two per transfer, hence this rule
+    // for the worst case; a pool on KV_PATH_AUTO applies the same threshold to the transfers each call
+    // actually needs, so lists whose host ids form runs or four-block lattices go staged at any block size.
     return 2 * blk_bytes >= KV_AUTO_MIN_TRANSFER ? KV_PATH_STAGED : KV_PATH_ZEROCOPY;
 }
 

@@ -176,8 +176,8 @@ def test_config5_full_shape_replay_2000_steps():
                          ids=["block8-random-2GB", "block64-contiguous-4GB", "block32-random-4GB", "block16-random-8GiB"])
 def test_config4_sweep_cells_at_full_payload(bs, contiguous, payload):
     """Cells of the block-size / fragmentation sweep at full payload, default path: 1 MiB blocks with random
-    tables (the zero-copy kernels), 8 MiB blocks with contiguous tables (long merged transfers), 4 MiB
-    blocks with random tables (uniform two-block transfers), and the cell of the paper's bandwidth table
+    tables (four-block lattices and pairs), 8 MiB blocks with contiguous tables (long merged transfers), 4 MiB
+    blocks with random tables, and the cell of the paper's bandwidth table
     (section 5.3.3): 2 MiB blocks, random tables, 8 GiB = 32768 tokens of 256 KB each way.  Each direction
     alone, then both at once."""
     w = W.config4_sweep_case(bs, contiguous, payload)
@@ -191,7 +191,6 @@ def test_config4_sweep_cells_at_full_payload(bs, contiguous, payload):
         t.rotate(r)
         moved = t.verify("swap-in alone, then both at once", n_read_back=4)
         assert moved == (r.n_in, r.n_out)
-        want = "zerocopy" if bs == 8 and not contiguous else "staged"
-        assert t.B.PATH_NAMES[t.pool.kv_get_stats()["last_path_out"]] == want
+        assert t.B.PATH_NAMES[t.pool.kv_get_stats()["last_path_out"]] == "staged"
     finally:
         t.close()

@@ -93,9 +93,9 @@ def test_long_runs_are_merged_and_cut_at_chunk_size():
     assert len(one) == 1 and one[0]["blocks_per_row"] == 64
     four, _ = check_plan(np.arange(77, 77 + 200), 512, 0)                    # larger, but fits one half: about four chunks,
     sizes = [_blocks(op) for op in four]                                     # the first of a swap-out half as long
-    assert 3 <= len({op["chunk"] for op in four}) <= 6 and sizes[0] == 25 and sizes[1] == 50
+    assert sizes == [26, 52, 52, 52, 18]                                     # equal chunks of a multiple of four blocks
     four_in, _ = check_plan(np.arange(77, 77 + 200), 512, 1)
-    assert [_blocks(op) for op in four_in] == [50, 50, 50, 50]
+    assert [_blocks(op) for op in four_in] == [52, 52, 52, 44]
 
 
 def test_short_runs_are_not_merged_into_uneven_transfers():
