@@ -30,6 +30,20 @@
         device time of every step's rotation, against the 70 ms a model step takes in the paper
         (section 5.3.4), i.e. how often the transfer would not hide behind the step.
 
+    python -m paper_2601_20309_b200.sweep lvf [--b-xfer N] [--steps K] [--out FILE]
+        Rotation lists made by the paper's Largest-VLT-First policy (section 4.2, Algorithm 1) on the serving
+        replay (8B shape, 8 requests/s, the paper's scheduler settings) under a transfer budget of N blocks:
+        device time of the first K steps that move blocks, against the 70 ms of a model step.  The policy
+        rotates hard; this shows what budget a PCIe link can hide.
+
+    python -m paper_2601_20309_b200.sweep lvf-table [--b-xfer N] [--steps K] [--eager-blocks E] [--out FILE]
+        The same replay and policy driven through the library's block table (kv_req_add / kv_req_append /
+        kv_eager_rotate / kv_req_rotate / kv_req_finish), which hands out the blocks itself: with E > 0 up
+        to E full blocks per step are copied to host memory in the background (the paper's eager block
+        rotation, section 4.3.2), so a preemption sends only what has no valid host copy and its device
+        blocks serve the requests resuming in the same rotation.  Reports, per step, the blocks moved at
+        rotation time and the rotation's device time, with and without the background copies.
+
     python -m paper_2601_20309_b200.sweep handoff [--out FILE]
         What a hand-off between the copy engine and a kernel costs while the host link is busy (plain torch
         streams, no library call): a host-to-device copy followed by a tiny kernel that waits for it, and a
@@ -276,6 +290,144 @@ def latency(out, block_size: int = 16) -> None:
               f"{r['zerocopy_us']} | {r['ce2d_us']} | {r['auto_over_best_pct']} % | {r['auto_untimed_us']} | {r['link_floor_us']} |")
 
 
+def lvf(out, b_xfer: int, n_steps: int) -> None:
+    import numpy as np
+    import torch
+    w = W.config5_lvf(rate=8.0, params=W.LVFParams(b_xfer=b_xfer))
+    shape = w.shape
+    moving = [r for r in w.steps if r.n_out + r.n_in][:n_steps]
+    dev = torch.empty(w.nb_gpu * shape.block_bytes, dtype=torch.uint8, device="cuda:0")
+    pool = B.KVPool(shape.num_layers, shape.block_size, shape.kv_heads, shape.head_dim, w.nb_gpu, w.nb_host,
+                    dev.data_ptr())
+    ms, blocks, outs = [], [], []
+    for r in moving:
+        pool.kv_rotate(r.out_gpu, r.out_host, r.in_host, r.in_gpu)
+        pool.kv_sync()
+        ms.append(pool.kv_get_stats()["last_union_ms"])
+        blocks.append(r.n_out + r.n_in)
+        outs.append(r.n_out)
+    pool.destroy()
+    ms, blocks, outs = np.array(ms), np.array(blocks), np.array(outs)
+    e = w.extra
+    rec = {"b_xfer": b_xfer, "steps_total": len(w.steps), "steps_that_move_blocks": int(sum(1 for r in w.steps if r.n_out + r.n_in)),
+           "steps_timed": len(ms), "blocks_per_step_median": float(np.median(blocks)), "blocks_per_step_max": int(blocks.max()),
+           "blocks_out_per_step_max": int(outs.max()), "ms_median": round(float(np.median(ms)), 2),
+           "ms_p99": round(float(np.percentile(ms, 99)), 2), "ms_max": round(float(ms.max()), 2),
+           "gbs_overall": round(float(blocks.sum() * shape.block_bytes / ms.sum() / 1e6), 1),
+           "steps_over_70ms": int((ms > 70.0).sum()), "share_over_70ms": round(float((ms > 70.0).mean()), 4),
+           "preempted_requests": int(e["preempted"].sum()), "resumed_requests": int(e["resumed"].sum()),
+           "admitted_requests": int(e["admitted"].sum()), "arrivals": int(e["arrivals"])}
+    _emit(rec, out)
+    print("\n| B_xfer | steps that move blocks (of 2000) | timed | blocks per step, median / max | ms median | ms p99 | ms max | GB/s overall | steps over 70 ms | requests preempted / resumed / admitted |\n|---|---|---|---|---|---|---|---|---|---|")
+    print(f"| {b_xfer} | {rec['steps_that_move_blocks']} | {rec['steps_timed']} | {rec['blocks_per_step_median']:.0f} / {rec['blocks_per_step_max']} | {rec['ms_median']} | "
+          f"{rec['ms_p99']} | {rec['ms_max']} | {rec['gbs_overall']} | {rec['steps_over_70ms']} ({100 * rec['share_over_70ms']:.1f} %) | "
+          f"{rec['preempted_requests']} / {rec['resumed_requests']} / {rec['admitted_requests']} |")
+
+
+def lvf_table(out, b_xfer: int, n_steps: int, eager_blocks: int) -> None:
+    import numpy as np
+    import torch
+    shape = W.SHAPE_8B
+    bs = shape.block_size
+    params = W.LVFParams(b_xfer=b_xfer)
+    # the arrivals, lengths and pool sizes of workload.config5_lvf (same seed, same draws)
+    rng = np.random.default_rng(W.MASTER_SEED + 6)
+    rate, duration_s, step_s, max_tokens = 8.0, 120.0, 0.070, 8192
+    n_arr = max(1, int(rng.poisson(rate * duration_s)))
+    arrive = np.sort(rng.uniform(0.0, duration_s, size=n_arr))
+    prompt = W.lognormal_tokens(rng, n_arr, 512, 1, max_tokens)
+    output = W.lognormal_tokens(rng, n_arr, 256, 1, max_tokens)
+    nblk = lambda tokens: -(-int(tokens) // bs)
+    a_step = np.floor(arrive / step_s).astype(np.int64)
+    horizon = int(a_step.max() + output.max() + 2)
+    delta = np.zeros(horizon + 1, np.int64)
+    for s_, p_, o_ in zip(a_step, prompt, output):
+        delta[s_] += nblk(p_ + o_)
+        delta[min(horizon, s_ + int(o_))] -= nblk(p_ + o_)
+    demand = int(np.cumsum(delta).max())
+    nb_gpu = max(int(0.40 * demand), nblk((prompt + output).max()) + 8)
+    nb_host = max(2 * demand, 64)
+    dev = torch.empty(nb_gpu * shape.block_bytes, dtype=torch.uint8, device="cuda:0")
+    pool = B.KVPool(shape.num_layers, shape.block_size, shape.kv_heads, shape.head_dim, nb_gpu, nb_host, dev.data_ptr())
+    table = B.KVTable(pool)
+    running, rotary, waiting, remaining = {}, {}, [], {}
+    ms, moved_out, moved_in, discarded, eager_sent, eager_ms = [], [], [], [], [], []
+    nxt, step = 0, 0
+    while len(ms) < n_steps and step < 2000:
+        t_now = step * step_s
+        while nxt < n_arr and a_step[nxt] <= step:
+            waiting.append(nxt)
+            nxt += 1
+        for rid in [r for r in running if remaining[r] <= 0]:
+            del running[rid]
+            table.kv_req_finish(rid)
+        info = {r: table.kv_req_info(r) for r in list(running) + list(rotary)}
+        grow_need = sum(1 for r in running if info[r]["tokens"] % bs == 0)
+        st0 = table.kv_table_get_stats()
+        b_hbm = max(0, st0["free_gpu_blocks"] - grow_need)
+        reqs = [(r, "running", W.vlt("running", t_now, t0, params), info[r]["num_blocks"]) for r, t0 in running.items()]
+        reqs += [(r, "waiting", W.vlt("waiting", t_now, float(arrive[r]), params), nblk(prompt[r])) for r in waiting]
+        reqs += [(r, "rotary", W.vlt("rotary", t_now, t0, params), info[r]["num_blocks"]) for r, t0 in rotary.items()]
+        preempt, prio = W.lvf_select(reqs, b_hbm, params.b_xfer)
+        resume = [r for r in prio if r in rotary]
+        admit = [r for r in prio if r not in rotary]
+        # the table lets resuming requests take what the preempted ones release; it refuses what does not fit
+        while True:
+            rc = table.kv_req_rotate(preempt, resume, check=False)
+            if rc == B.KV_OK or not resume:
+                break
+            resume.pop()
+        if rc != B.KV_OK:
+            raise RuntimeError(f"kv_req_rotate failed: {rc}")
+        pool.kv_sync()
+        st1 = table.kv_table_get_stats()
+        out_b = st1["preempt_blocks_moved"] - st0["preempt_blocks_moved"]
+        in_b = st1["resume_blocks_moved"] - st0["resume_blocks_moved"]
+        if out_b + in_b:
+            ms.append(pool.kv_get_stats()["last_union_ms"])
+            moved_out.append(out_b)
+            moved_in.append(in_b)
+            discarded.append(st1["discarded_blocks"] - st0["discarded_blocks"])
+        for rid in preempt:
+            del running[rid]
+            rotary[rid] = t_now
+        for rid in resume:
+            del rotary[rid]
+            running[rid] = t_now
+        for rid in admit:
+            if table.kv_req_add(rid, int(prompt[rid]), check=False) == B.KV_OK:
+                waiting.remove(rid)
+                remaining[rid] = int(output[rid])
+                running[rid] = t_now
+        for rid in running:
+            if table.kv_req_append(rid, 1, check=False) == B.KV_OK:
+                remaining[rid] -= 1
+        if eager_blocks > 0:
+            n_sent = table.kv_eager_rotate(eager_blocks)
+            pool.kv_sync()
+            if n_sent:
+                eager_sent.append(n_sent)
+                eager_ms.append(pool.kv_get_stats()["last_union_ms"])
+        step += 1
+    table.destroy()
+    pool.destroy()
+    ms, mo, mi, dc = (np.array(x, float) for x in (ms, moved_out, moved_in, discarded))
+    rec = {"b_xfer": b_xfer, "eager_blocks_per_step": eager_blocks, "steps_run": step, "rotations_timed": len(ms),
+           "blocks_out_per_rotation_median": float(np.median(mo)), "blocks_in_per_rotation_median": float(np.median(mi)),
+           "blocks_discarded_per_rotation_median": float(np.median(dc)),
+           "blocks_out_total": int(mo.sum()), "blocks_discarded_total": int(dc.sum()), "blocks_in_total": int(mi.sum()),
+           "rotation_ms_median": round(float(np.median(ms)), 2), "rotation_ms_p99": round(float(np.percentile(ms, 99)), 2),
+           "rotation_ms_max": round(float(ms.max()), 2), "rotations_over_70ms": int((ms > 70.0).sum()),
+           "background_blocks_total": int(np.sum(eager_sent)) if eager_sent else 0,
+           "background_ms_median": round(float(np.median(eager_ms)), 2) if eager_ms else None}
+    _emit(rec, out)
+    print("\n| B_xfer | background blocks per step | rotations timed | blocks out / discarded / in per rotation (median) | blocks out / discarded / in, total | "
+          "rotation ms median | p99 | max | over 70 ms | background copies: blocks, median ms per step |\n|---|---|---|---|---|---|---|---|---|---|")
+    print(f"| {b_xfer} | {eager_blocks} | {rec['rotations_timed']} | {rec['blocks_out_per_rotation_median']:.0f} / {rec['blocks_discarded_per_rotation_median']:.0f} / "
+          f"{rec['blocks_in_per_rotation_median']:.0f} | {rec['blocks_out_total']} / {rec['blocks_discarded_total']} / {rec['blocks_in_total']} | {rec['rotation_ms_median']} | "
+          f"{rec['rotation_ms_p99']} | {rec['rotation_ms_max']} | {rec['rotations_over_70ms']} | {rec['background_blocks_total']}, {rec['background_ms_median']} |")
+
+
 def handoff(out) -> None:
     import torch
     dev = "cuda:0"
@@ -385,7 +537,9 @@ def budget(out, b_xfer: int) -> None:
 
 def main() -> None:
     ap = argparse.ArgumentParser()
-    ap.add_argument("what", choices=["probe", "paths", "overlap", "latency", "budget", "handoff"])
+    ap.add_argument("what", choices=["probe", "paths", "overlap", "latency", "budget", "handoff", "lvf", "lvf-table"])
+    ap.add_argument("--eager-blocks", type=int, default=0, help="lvf-table: full blocks copied out in the background per step")
+    ap.add_argument("--steps", type=int, default=300, help="lvf: steps to time")
     ap.add_argument("--out", default=None)
     ap.add_argument("--max-payload-gb", type=float, default=4.0)
     ap.add_argument("--b-xfer", type=int, default=2400, help="budget: blocks per step, both directions together")
@@ -407,6 +561,10 @@ def main() -> None:
         latency(out, a.block_size)
     elif a.what == "handoff":
         handoff(out)
+    elif a.what == "lvf":
+        lvf(out, a.b_xfer, a.steps)
+    elif a.what == "lvf-table":
+        lvf_table(out, a.b_xfer, a.steps, a.eager_blocks)
     else:
         budget(out, a.b_xfer)
 
