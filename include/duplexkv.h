@@ -60,7 +60,7 @@ extern "C" {
 /* transfer paths (how the host link is driven) */
 #define KV_PATH_AUTO          0     /* per call.  8 MiB or less per direction (2 MiB for blocks under 2 MiB):
                                        CE2D, the lowest fixed cost.  Larger calls: STAGED when the
-                                       copy-engine transfers the call needs would average 3 MiB or more,
+                                       copy-engine transfers the call needs would average 2.5 MiB or more,
                                        else ZEROCOPY (see kv_path_for)                                   */
 #define KV_PATH_ZEROCOPY      1     /* SM kernels read/write mapped pinned host memory directly          */
 #define KV_PATH_STAGED        2     /* pack kernel -> contiguous HBM staging -> copy engine (and reverse)*/

@@ -21,7 +21,7 @@ namespace {
 
 constexpr int KV_SLOTS = 8;            // descriptor / event ring depth per direction
 constexpr int KV_MAX_CE_STREAMS = 4;
-constexpr int64_t KV_AUTO_MIN_TRANSFER = 3ll << 20;   // AUTO: staged when its transfers average 3 MiB or more
+constexpr int64_t KV_AUTO_MIN_TRANSFER = 5ll << 19;   // AUTO: staged when its transfers average 2.5 MiB or more
 // AUTO, calls bound by fixed costs rather than by the link (measured on scattered ids, call to completion):
 // one copy-engine transfer per block is the quickest up to 8 MiB per direction of 2 MiB blocks (65 / 111 /
 // 212 us for 1 / 2 / 4 blocks each way against 85 / 141 / 231 us staged and 87 / 143 / 247 us for the
@@ -441,8 +441,8 @@ std::vector<int64_t> chunk_bounds(int64_t n, int64_t first, int64_t chunk, bool 
 // (a, a+g, a+kg, a+kg+g) are one 3-D copy-engine transfer: two rows g blocks apart, two slices k rows apart,
 // and a transfer of four blocks runs at the rate of one twice as long as a pair's (measured both ways: 97
 // against 94 GB/s for 2 MiB blocks).  Two pairs (x, x+g) and (x', x'+g) form such a lattice exactly when
-// their starts are congruent modulo g, so one sweep over the sorted ids keeps, per (g, x mod g), the latest
-// pair still waiting for a partner and closes a lattice whenever a second one turns up: a few probes per
+// their starts are congruent modulo g, so one sweep over the sorted ids keeps, per (g, x mod g), one pair
+// still waiting for a partner and closes a lattice whenever a second one turns up: a few probes per
 // block, and about three quarters of a uniformly scattered list find a place (95 % of a denser one).  The
 // blocks left over travel as before, two per transfer.  `order` comes in sorted by host id and leaves as the
 // staging order: the blocks of each transfer next to one another, transfers in issue order (lattices first).
@@ -481,12 +481,14 @@ bool plan_lattices(const PlanParams &pp, const int32_t *host_ids, int64_t n, int
             size_t h = (size_t)((key * 0x9E3779B97F4A7C15ull) >> (64 - bits));
             while (table[h].key != ~0ull && table[h].key != key) h = (h + 1) & (cap - 1);
             Slot &w = table[h];
-            if (w.key == key && w.i >= 0 && !used[(size_t)w.i] && !used[(size_t)w.j] && x - hid(w.i) >= 2 * g) {
+            const bool waiting = w.key == key && w.i >= 0 && !used[(size_t)w.i] && !used[(size_t)w.j];
+            if (waiting && x - hid(w.i) >= 2 * g) {
                 quads.push_back(Quad{{w.i, w.j, (int32_t)i, (int32_t)j}, g, (x - hid(w.i)) / g});
                 used[(size_t)w.i] = used[(size_t)w.j] = used[(size_t)i] = used[(size_t)j] = 1;
                 w.i = w.j = -1;
                 break;
             }
+            if (waiting) continue;       // the waiting pair ends where this one starts (an arithmetic run): it keeps waiting
             w.key = key;
             w.i = (int32_t)i;
             w.j = (int32_t)j;
@@ -1092,7 +1094,7 @@ int32_t kv_path_for(int64_t blk_bytes)
 {
     // Measured on B200 behind PCIe Gen5 x16, both directions busy: a copy-engine transfer costs a fixed
     // start-up (about 10 us with the other direction busy) plus its bytes, so the staged path wins once its
-    // transfers carry 3 MiB or more; below that the zero-copy kernels, which pay no per-transfer cost,
+    // transfers carry 2.5 MiB or more; below that the zero-copy kernels, which pay no per-transfer cost,
     // are ahead.  Blocks with no neighbours in host memory travel at least two per transfer, hence this rule
     // for the worst case; a pool on KV_PATH_AUTO applies the same threshold to the transfers each call
     // actually needs, so lists whose host ids form runs or four-block lattices go staged at any block size.

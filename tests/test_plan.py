@@ -138,3 +138,16 @@ def test_other_block_sizes(blk):
     rng = np.random.default_rng(9)
     check_plan(rng.choice(5000, 333, replace=False), max(2, (64 << 20) // blk), 0, blk=blk)
     check_plan(np.arange(10, 410), max(2, (64 << 20) // blk), 1, blk=blk)
+
+
+def test_lattices_with_repeated_sources_and_dense_ids():
+    """Swap-in sources may repeat: the plan must still name every list entry exactly once; and a dense
+    scattered list (every other id) is all lattices."""
+    rng = np.random.default_rng(5)
+    ids = rng.choice(3000, 300, replace=False)
+    ids = np.concatenate([ids, ids[:40], ids[:7]])                           # 47 entries repeat earlier ones
+    check_plan(rng.permutation(ids), 512, 1)
+    ops, _ = check_plan(np.arange(0, 400, 2), 512, 0)                        # 0, 2, 4, ...: gap 2 everywhere
+    assert all(_blocks(op) == 4 for op in ops)
+    ops, _ = check_plan(np.arange(0, 64, 2), 3, 0)                           # halves too small for a lattice: pairs
+    assert all(op["slices"] == 1 for op in ops)

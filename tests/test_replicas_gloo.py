@@ -75,3 +75,19 @@ def test_rank_environment():
     env = R.rank_env(3, 8, 29511, base={"KEEP": "1"})
     assert env == {"KEEP": "1", "RANK": "3", "LOCAL_RANK": "3", "WORLD_SIZE": "8", "LOCAL_WORLD_SIZE": "8",
                    "MASTER_ADDR": "127.0.0.1", "MASTER_PORT": "29511"}
+
+
+def test_bench_gpus_flag_starts_that_many_replicas():
+    """`python bench.py --gpus 2` without a launcher must start two ranks itself.  On a machine without a
+    GPU each rank stops with the no-fallback message, which is enough to count them."""
+    import subprocess
+    import sys
+    if torch.cuda.is_available():
+        pytest.skip("counts ranks by their no-GPU message; covered by the stub test on a GPU box")
+    root = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+    env = {k: v for k, v in os.environ.items() if k not in ("RANK", "LOCAL_RANK", "WORLD_SIZE", "MASTER_ADDR", "MASTER_PORT")}
+    res = subprocess.run([sys.executable, os.path.join(root, "bench.py"), "--gpus", "2", "--steps", "1"],
+                         capture_output=True, text=True, env=env, timeout=600)
+    assert res.returncode != 0
+    assert res.stderr.count("needs a CUDA device") == 2
+    assert res.stdout.strip() == ""
