@@ -215,9 +215,10 @@ int32_t kv_rotate_req(kv_pool_t *pool,
  * What copy-engine transfers the STAGED path would make for one direction of a call (no pool, no GPU).
  * Where the host ids form long runs (8 blocks and more on average) the list is taken in ascending order
  * of host id, each run is one transfer and equal runs at a constant spacing share one strided transfer.
- * Otherwise every block counts as a single: four blocks whose ids form a 2 x 2 lattice (a, a+g, a+kg,
- * a+kg+g) share one 3-D transfer, the blocks left over travel two per transfer (neighbours in ascending
- * order, any distance apart in host memory), lattices first -- transfers of few sizes keep the two copy
+ * Otherwise every block counts as a single: four blocks (of less than 4 MiB) whose ids form a 2 x 2
+ * lattice (a, a+g, a+kg, a+kg+g) share one 3-D transfer, the blocks left over travel two per transfer
+ * (neighbours in ascending order, any distance apart in host memory), lattices first; blocks of 4 MiB and
+ * more travel two per transfer throughout -- transfers of few sizes keep the two copy
  * engines of a rotation in step (section 4.3.2's "merge small segments into large transfers", bounded
  * here by what the ids allow).  The sequence is cut into chunks of at most half_blocks blocks (one
  * staging half each; about four chunks for a call that would fit one half, a single chunk for a call of

@@ -33,6 +33,7 @@ constexpr int64_t KV_AUTO_TINY_BYTES = 8ll << 20;
 constexpr int64_t KV_AUTO_TINY_BYTES_SMALL_BLOCKS = 2ll << 20;
 constexpr int64_t KV_MERGE_MIN_MEAN_RUN = 8;
 constexpr int64_t KV_QUAD_MAX_GAP = 256;              // STAGED, scattered ids: largest row gap (blocks) of a four-block lattice
+constexpr int64_t KV_QUAD_ENOUGH_BYTES = 8ll << 20;  //         no lattices when a pair of blocks already carries this much
 constexpr int KV_QUAD_PARTNERS = 6;                   //         partners tried per block when looking for lattices
 constexpr int64_t KV_PLAN_CHUNKS = 4;                 // STAGED: a call that fits one staging half is still cut into about this many chunks ...
 constexpr int64_t KV_PLAN_ONE_CHUNK_BYTES = 128ll << 20;   // ... unless it moves this much or less per direction: then it is one chunk          // STAGED: merge runs of host ids when they average 8 blocks or more
@@ -453,7 +454,9 @@ bool plan_lattices(const PlanParams &pp, const int32_t *host_ids, int64_t n, int
     const std::vector<int32_t> sorted = order;
     auto hid = [&](int64_t q) { return (int64_t)host_ids[sorted[(size_t)q]]; };
     const int64_t gmax = std::min<int64_t>(KV_QUAD_MAX_GAP, pp.max_pitch / pp.blk);
-    if (gmax < 1 || chunk < 4 || n < 8) return false;
+    // blocks of 4 MiB and more already travel in pairs of 8 MiB and more, which run at the link's rate:
+    // lattices would only add a second transfer size (measured with 8 MiB blocks: 92 GB/s against 96-99)
+    if (gmax < 1 || chunk < 4 || n < 8 || 2 * pp.blk >= KV_QUAD_ENOUGH_BYTES) return false;
     struct Slot {
         uint64_t key;
         int32_t i, j;

@@ -151,3 +151,12 @@ def test_lattices_with_repeated_sources_and_dense_ids():
     assert all(_blocks(op) == 4 for op in ops)
     ops, _ = check_plan(np.arange(0, 64, 2), 3, 0)                           # halves too small for a lattice: pairs
     assert all(op["slices"] == 1 for op in ops)
+
+
+def test_large_blocks_travel_in_pairs_only():
+    """A pair of 4 MiB blocks is an 8 MiB transfer already: no lattices, one transfer size."""
+    rng = np.random.default_rng(12)
+    ids = rng.choice(20_000, 600, replace=False)
+    for blk, expect_fours in ((1 << 20, True), (2 << 20, True), (4 << 20, False), (5 << 20, False), (8 << 20, False)):
+        ops, _ = check_plan(ids, 4096, 0, blk=blk)
+        assert any(_blocks(op) == 4 for op in ops) == expect_fours, blk
