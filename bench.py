@@ -628,6 +628,9 @@ def main() -> None:
         args.warmup = 3
     if args.gpus > 1 and "WORLD_SIZE" not in os.environ and args.impl == "ours":
         # not started by a launcher: start the N replicas here, one process per GPU
+        import torch
+        if torch.cuda.is_available() and torch.cuda.device_count() < args.gpus:
+            raise SystemExit(f"bench.py: --gpus {args.gpus} asked for, the node has {torch.cuda.device_count()} GPUs")
         from paper_2601_20309_b200 import replicas as R
         sys.exit(R.main_spawn(args.gpus))
     rank = int(os.environ.get("RANK", "0"))

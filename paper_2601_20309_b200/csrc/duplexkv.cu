@@ -37,9 +37,13 @@ constexpr int64_t KV_QUAD_ENOUGH_BYTES = 8ll << 20;  //         no lattices when
 constexpr int KV_QUAD_PARTNERS = 6;                   //         partners tried per block when looking for lattices
 constexpr int64_t KV_PLAN_CHUNKS = 4;                 // STAGED: a call that fits one staging half is still cut into about this many chunks ...
 constexpr int64_t KV_PLAN_ONE_CHUNK_BYTES = 128ll << 20;   // ... unless it moves this much or less per direction: then it is one chunk          // STAGED: merge runs of host ids when they average 8 blocks or more
+// HBM-to-HBM shape of the bulk kernel's ring.  Measured on the 3.87 GB gather (148 CTAs): the rate peaks with
+// about 32 KiB of loads in flight per SM and falls with more -- 16 KiB x 2 ahead 6.42-6.45 TB/s, 32 KiB x 1
+// ahead 6.43, 8 KiB x 5 ahead 6.40, 16 KiB x 3 ahead 6.32, 16 KiB x 5 ahead (the first choice) 6.09-6.15, one
+// load ahead 5.56; 4 KiB copies are bound by the one thread that issues them (3.8); two CTAs per SM lose 5 %.
 constexpr int BULK_STAGE = 16384;      // bytes per shared-memory stage of the bulk kernel
-constexpr int BULK_NS = 8;             // stages
-constexpr int BULK_AHEAD = 5;          // loads in flight ahead of the stores
+constexpr int BULK_NS = 4;             // stages
+constexpr int BULK_AHEAD = 2;          // loads in flight ahead of the stores
 // the same kernel when one side is mapped host memory: the link needs far fewer bytes in flight than
 // HBM does, and a small shared-memory footprint leaves the SMs' L1 to whatever else runs on them
 constexpr int LINK_STAGE = 8192;
