@@ -42,7 +42,7 @@ WORKLOAD = ("config2 llama-3-8b-shaped KV (32 layers, 8 kv heads, head_dim 128, 
             "paired rotate of %d requests each way per step")
 # DRAM traffic of one pack / unpack launch, from the ncu capture of an 88-block (184.55 MB) launch on the
 # --small case (retaken after the kernel's last change: same figures): dram__bytes_read.sum = 1.0001 x
-# payload (no byte read twice); dram__bytes_write.sum = payload - 48 to 50 MB, the lines still in L2 when the
+# payload (no byte read twice); dram__bytes_write.sum = payload - 45 to 50 MB, the lines still in L2 when the
 # kernel ends.  Reads scale with the payload, the L2 tail does not.
 def ncu_traffic_per_launch(payload_bytes: float) -> float:
     return 1.00005 * payload_bytes + max(0.0, payload_bytes - 48.5e6)
