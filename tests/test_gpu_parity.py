@@ -579,3 +579,40 @@ def test_lists_made_by_the_lvf_scheduler_match_the_oracle():
         p.assert_equal("LVF final")
     finally:
         p.close()
+
+
+@pytest.mark.parametrize("seed", range(12))
+def test_random_shapes_lists_and_staging_sizes(seed):
+    """Seeded random cases across shapes, pool sizes, list lengths, staging sizes (so that the staged plan
+    is cut into one to many chunks, with four-block lattices, pairs and singles in them), paths and host
+    layouts: three calls queued without syncing, then both pools against the oracle."""
+    rng = np.random.default_rng(1000 + seed)
+    shape = W.KVShape(int(rng.choice([1, 2, 3, 5])), int(rng.choice([8, 16, 32])), int(rng.choice([1, 2, 8])), int(rng.choice([64, 128])))
+    nbg, nbh = int(rng.integers(60, 260)), int(rng.integers(80, 400))
+    path = int(rng.choice([0, 2, 2, 1]))
+    layout = int(rng.choice([0, 0, 1]))
+    staging = int(rng.choice([2, 5, 8, 16, 33, 1000])) * shape.block_bytes
+    p = _pair(shape, nbg, nbh, seed=seed, path=path, host_layout=layout, staging_bytes=staging)
+    try:
+        for call in range(3):
+            n_out = int(rng.integers(1, min(nbg, nbh) // 2))
+            n_in = int(rng.integers(1, min(nbg, nbh) // 2))
+            og = rng.choice(nbg, n_out, replace=False).astype(np.int32)
+            oh = rng.choice(nbh, n_out, replace=False).astype(np.int32)
+            ig = np.setdiff1d(np.arange(nbg), og)
+            ig = rng.choice(ig, min(n_in, len(ig)), replace=False).astype(np.int32)
+            ih = np.setdiff1d(np.arange(nbh), oh)
+            ih = rng.choice(ih, len(ig), replace=True).astype(np.int32)         # swap-in sources may repeat
+            if call == 1 and rng.random() < 0.5:                                  # every other host id: all lattices
+                oh = (2 * np.arange(n_out) % nbh).astype(np.int32)
+                oh = np.unique(oh)[:n_out]
+                og = og[:len(oh)]
+                ih = np.setdiff1d(np.arange(nbh), oh)
+                ih = rng.choice(ih, len(ig), replace=True).astype(np.int32) if len(ih) else ih[:0].astype(np.int32)
+                ig = ig[:len(ih)]
+            r = W.Rotation(og, oh, ih, ig, np.zeros(1), np.zeros(1))
+            assert p.rotate_both(r) == 0, (seed, call)
+        p.assert_equal(f"random case {seed}: shape {shape}, pools {nbg}/{nbh}, path {path}, layout {layout}, staging {staging}")
+        assert p.pool.kv_get_stats()["device_status"] == 0
+    finally:
+        p.close()
