@@ -52,6 +52,18 @@ constexpr int LINK_AHEAD = 6;
 // other shapes of the same ring for the link (kv_pool_config_t.link_variant 1 and 2): fewer, larger bulk copies
 constexpr int LINK1_STAGE = 32768, LINK1_NS = 4, LINK1_AHEAD = 2;
 constexpr int LINK2_STAGE = 65536, LINK2_NS = 3, LINK2_AHEAD = 1;
+// Small segments (the shard of one rank under tensor parallelism, small block sizes): an item is a whole
+// segment, so with the large ring too few bytes are in flight and one thread issues too few copies per
+// second (measured on a 2 GiB gather: 5.1 / 3.4 / 1.8 / 0.9 TB/s for segments of 8 / 4 / 2 / 1 KiB against 6.4
+// for 16 KiB and more).  Such launches take a ring of smaller stages per warp and more issuing warps per
+// CTA.  HBM to HBM, what counts is many warps with few loads ahead each, 32 KiB in flight per SM as in the
+// large ring: 2 / 4 / 8 warps x 2 ahead reach 6.43 / 6.24 / 5.98 TB/s at 8 / 4 / 2 KiB and 16 warps x 1 ahead
+// 6.04 at 1 KiB, while 4 or 8 loads ahead on half as many warps stay at 4.9-5.0.  Over the link every shape
+// with 48 KiB in flight per CTA reaches the zero-copy ceiling (80.4-80.7 GB/s both ways, where the 8 KiB ring
+// gave 79.5 / 74.2 / 63.5 at 4 / 2 / 1 KiB).
+constexpr int SMALL_NS = 4, SMALL_AHEAD = 2;           // HBM to HBM: stages of 8 / 4 / 2 KiB on 2 / 4 / 8 warps
+constexpr int TINY_NS = 3, TINY_AHEAD = 1;             //             stages of 1 KiB on 16 warps
+constexpr int SMALL_LINK_NS = 8, SMALL_LINK_AHEAD = 6; // over the link: stages of 4 / 2 / 1 KiB on 2 / 4 / 8 warps
 constexpr int LDST_THREADS = 512;
 constexpr int LDST_UNROLL = 4;         // 512 threads * 4 * 16 B = 32 KiB per item
 constexpr int LDST_CHUNK = LDST_THREADS * LDST_UNROLL * 16;
@@ -230,6 +242,64 @@ int clamp_ctas(const KvJob &job, const KvDir &d, int want)
     return (int)std::max<long long>(1, std::min<long long>(want, items));
 }
 
+// one shape of the bulk kernel: ring geometry and issuing warps per CTA
+template <int STAGE, int NS, int AHEAD, int WARPS>
+struct Bulk {
+    static_assert(WARPS >= 1 && WARPS <= KV_BULK_MAX_WARPS, "issuing warps per CTA");
+    static constexpr int smem = STAGE * NS * WARPS;
+    static cudaError_t prepare()
+    {
+        return cudaFuncSetAttribute(kv_copy_bulk<STAGE, NS, AHEAD>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+    }
+    static void launch(int grid, cudaStream_t stream, const KvJob &job)
+    {
+        kv_copy_bulk<STAGE, NS, AHEAD><<<grid, 32 * WARPS, smem, stream>>>(job);
+    }
+};
+using BulkHbm = Bulk<BULK_STAGE, BULK_NS, BULK_AHEAD, 1>;
+using BulkHbm8k = Bulk<8192, SMALL_NS, SMALL_AHEAD, 2>;
+using BulkHbm4k = Bulk<4096, SMALL_NS, SMALL_AHEAD, 4>;
+using BulkHbm2k = Bulk<2048, SMALL_NS, SMALL_AHEAD, 8>;
+using BulkHbm1k = Bulk<1024, TINY_NS, TINY_AHEAD, 16>;
+using BulkLink = Bulk<LINK_STAGE, LINK_NS, LINK_AHEAD, 1>;
+using BulkLink1 = Bulk<LINK1_STAGE, LINK1_NS, LINK1_AHEAD, 1>;
+using BulkLink2 = Bulk<LINK2_STAGE, LINK2_NS, LINK2_AHEAD, 1>;
+using BulkLink4k = Bulk<4096, SMALL_LINK_NS, SMALL_LINK_AHEAD, 2>;
+using BulkLink2k = Bulk<2048, SMALL_LINK_NS, SMALL_LINK_AHEAD, 4>;
+using BulkLink1k = Bulk<1024, SMALL_LINK_NS, SMALL_LINK_AHEAD, 8>;
+
+cudaError_t prepare_bulk_kernels()
+{
+    cudaError_t (*const all[])() = {BulkHbm::prepare,   BulkHbm8k::prepare,  BulkHbm4k::prepare,  BulkHbm2k::prepare,
+                                    BulkHbm1k::prepare, BulkLink::prepare,   BulkLink1::prepare,  BulkLink2::prepare,
+                                    BulkLink4k::prepare, BulkLink2k::prepare, BulkLink1k::prepare};
+    for (auto fn : all) {
+        const cudaError_t rc = fn();
+        if (rc != cudaSuccess) return rc;
+    }
+    return cudaSuccess;
+}
+
+// the bulk kernel's shape for items of job.chunk bytes
+void launch_bulk(const kv_pool *p, const KvJob &job, int grid, cudaStream_t stream, bool link)
+{
+    const int c = job.chunk;
+    if (link) {
+        if (c <= 1024) BulkLink1k::launch(grid, stream, job);
+        else if (c <= 2048) BulkLink2k::launch(grid, stream, job);
+        else if (c <= 4096) BulkLink4k::launch(grid, stream, job);
+        else if (p->cfg.link_variant == 1) BulkLink1::launch(grid, stream, job);
+        else if (p->cfg.link_variant == 2) BulkLink2::launch(grid, stream, job);
+        else BulkLink::launch(grid, stream, job);
+    } else {
+        if (c <= 1024) BulkHbm1k::launch(grid, stream, job);
+        else if (c <= 2048) BulkHbm2k::launch(grid, stream, job);
+        else if (c <= 4096) BulkHbm4k::launch(grid, stream, job);
+        else if (c <= 8192) BulkHbm8k::launch(grid, stream, job);
+        else BulkHbm::launch(grid, stream, job);
+    }
+}
+
 cudaError_t launch_job(kv_pool *p, const KvJob &job, cudaStream_t stream, bool link = false)
 {
     const int grid = job.dir[0].ctas + job.dir[1].ctas;
@@ -237,14 +307,8 @@ cudaError_t launch_job(kv_pool *p, const KvJob &job, cudaStream_t stream, bool l
     if (use_ldst(p)) {
         if (ldst32(p, link)) kv_copy_ldst<LDST_THREADS, LDST32_UNROLL, 32><<<grid, LDST_THREADS, 0, stream>>>(job);
         else kv_copy_ldst<LDST_THREADS, LDST_UNROLL, 16><<<grid, LDST_THREADS, 0, stream>>>(job);
-    } else if (link && p->cfg.link_variant == 1) {
-        kv_copy_bulk<LINK1_STAGE, LINK1_NS, LINK1_AHEAD><<<grid, 32, LINK1_STAGE * LINK1_NS, stream>>>(job);
-    } else if (link && p->cfg.link_variant == 2) {
-        kv_copy_bulk<LINK2_STAGE, LINK2_NS, LINK2_AHEAD><<<grid, 32, LINK2_STAGE * LINK2_NS, stream>>>(job);
-    } else if (link) {
-        kv_copy_bulk<LINK_STAGE, LINK_NS, LINK_AHEAD><<<grid, 32, LINK_STAGE * LINK_NS, stream>>>(job);
     } else {
-        kv_copy_bulk<BULK_STAGE, BULK_NS, BULK_AHEAD><<<grid, 32, BULK_STAGE * BULK_NS, stream>>>(job);
+        launch_bulk(p, job, grid, stream, link);
     }
     p->stats.kernel_launches++;
     return cudaGetLastError();
@@ -1269,14 +1333,7 @@ int32_t kv_pool_create(const kv_pool_config_t *cfg, kv_pool_t **out)
             KV_CREATE_CUDA(cudaEventCreateWithFlags(&s.join_ev[k], cudaEventDisableTiming));
         }
     }
-    KV_CREATE_CUDA(cudaFuncSetAttribute(kv_copy_bulk<BULK_STAGE, BULK_NS, BULK_AHEAD>,
-                                        cudaFuncAttributeMaxDynamicSharedMemorySize, BULK_STAGE * BULK_NS));
-    KV_CREATE_CUDA(cudaFuncSetAttribute(kv_copy_bulk<LINK_STAGE, LINK_NS, LINK_AHEAD>,
-                                        cudaFuncAttributeMaxDynamicSharedMemorySize, LINK_STAGE * LINK_NS));
-    KV_CREATE_CUDA(cudaFuncSetAttribute(kv_copy_bulk<LINK1_STAGE, LINK1_NS, LINK1_AHEAD>,
-                                        cudaFuncAttributeMaxDynamicSharedMemorySize, LINK1_STAGE * LINK1_NS));
-    KV_CREATE_CUDA(cudaFuncSetAttribute(kv_copy_bulk<LINK2_STAGE, LINK2_NS, LINK2_AHEAD>,
-                                        cudaFuncAttributeMaxDynamicSharedMemorySize, LINK2_STAGE * LINK2_NS));
+    KV_CREATE_CUDA(prepare_bulk_kernels());
 #undef KV_CREATE_CUDA
 
     try {
@@ -1965,8 +2022,7 @@ extern "C" int32_t kv_gather_blocks_static(const void *device_base, int32_t num_
         // once per device, with that device current
         void *ptr = nullptr;
         KV_CUDA(nullptr, cudaGetSymbolAddress((void **)&ptr, kv_static_scratch));
-        KV_CUDA(nullptr, cudaFuncSetAttribute(kv_copy_bulk<BULK_STAGE, BULK_NS, BULK_AHEAD>,
-                                              cudaFuncAttributeMaxDynamicSharedMemorySize, BULK_STAGE * BULK_NS));
+        KV_CUDA(nullptr, BulkHbm::prepare());
         g_static_scratch[dev] = ptr;
     }
     int2 *pairs = (int2 *)g_static_scratch[dev];
@@ -1997,7 +2053,7 @@ extern "C" int32_t kv_gather_blocks_static(const void *device_base, int32_t num_
     kd.src_blocks = (int)num_gpu_blocks;
     kd.dst_blocks = (int)n;
     kd.ctas = clamp_ctas(job, kd, sm_count > 0 ? sm_count : 1);
-    kv_copy_bulk<BULK_STAGE, BULK_NS, BULK_AHEAD><<<kd.ctas, 32, BULK_STAGE * BULK_NS, st>>>(job);
+    BulkHbm::launch(kd.ctas, st, job);
     KV_CUDA(nullptr, cudaGetLastError());
     unsigned int seen = 0;
     KV_CUDA(nullptr, cudaMemcpyAsync(&seen, status, sizeof(seen), cudaMemcpyDeviceToHost, st));

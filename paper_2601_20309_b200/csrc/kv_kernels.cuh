@@ -11,10 +11,10 @@
 // through consecutive destination addresses and re-reads the pair list only when it moves to the
 // next block.
 //
-// kv_copy_bulk  one thread per CTA drives bulk asynchronous copies (global -> shared -> global)
-//               through a ring of shared-memory stages guarded by mbarriers; no registers or
-//               warps are spent on the payload.  Used for HBM<->HBM gather/scatter and for
-//               HBM<->mapped host memory.
+// kv_copy_bulk  one thread per warp drives bulk asynchronous copies (global -> shared -> global)
+//               through a ring of shared-memory stages guarded by mbarriers; no registers are
+//               spent on the payload.  One warp per CTA when segments are large, up to 16 when
+//               they are small.  Used for HBM<->HBM gather/scatter and for HBM<->mapped host memory.
 // kv_copy_ldst  every thread moves 16-byte (or 32-byte) vectors with streaming loads/stores, all loads of a
 //               chunk issued before its stores; each warp walks the pair list cooperatively
 //               (one coalesced load of up to 32 pairs, then shuffles).
@@ -233,22 +233,34 @@ __device__ __forceinline__ void kv_fence_mbar_init() { asm volatile("fence.mbarr
 // Stage s is refilled only after the store that last read it has finished reading: stores are
 // committed one group per item, in order, so allowing NS-AHEAD-1 newer groups to be pending
 // guarantees that.
+// The first thread of every warp of the CTA runs such a ring of its own (its own stages and barriers)
+// over its share of the CTA's items: one warp when the items are large, several when segments are
+// small, where one thread cannot issue copies fast enough and AHEAD small items are too few bytes in
+// flight.  Dynamic shared memory: STAGE * NS bytes per warp.
+#define KV_BULK_MAX_WARPS 16
 template <int STAGE, int NS, int AHEAD>
-__global__ void __launch_bounds__(32, 1) kv_copy_bulk(const __grid_constant__ KvJob job)
+__global__ void __launch_bounds__(32 * KV_BULK_MAX_WARPS, 1) kv_copy_bulk(const __grid_constant__ KvJob job)
 {
     static_assert(AHEAD >= 1 && AHEAD < NS, "AHEAD must be in [1, NS)");
     extern __shared__ __align__(128) unsigned char kv_smem[];
-    __shared__ __align__(8) unsigned long long full_bar[NS];
-    if (threadIdx.x != 0) return;
+    __shared__ __align__(8) unsigned long long full_bar[KV_BULK_MAX_WARPS][NS];
+    if ((threadIdx.x & 31) != 0) return;
+    const int warp = (int)(threadIdx.x >> 5), nwarps = (int)(blockDim.x >> 5);
 
     int dsel;
     long long lo, hi;
     if (!kv_my_range(job, dsel, lo, hi)) return;
+    {
+        const long long span = hi - lo;
+        hi = lo + span * (warp + 1) / nwarps;
+        lo = lo + span * warp / nwarps;
+        if (hi <= lo) return;
+    }
     const KvDir &d = job.dir[dsel];
     if (job.t_first) atomicMin(job.t_first, kv_globaltimer());
 
-    const uint32_t smem0 = kv_smem_u32(kv_smem);
-    const uint32_t bar0 = kv_smem_u32(full_bar);
+    const uint32_t smem0 = kv_smem_u32(kv_smem) + (uint32_t)warp * (uint32_t)(STAGE * NS);
+    const uint32_t bar0 = kv_smem_u32(full_bar[warp]);
 #pragma unroll
     for (int s = 0; s < NS; ++s) kv_mbar_init(bar0 + 8 * s, 1);
     kv_fence_mbar_init();

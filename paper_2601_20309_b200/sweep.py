@@ -114,18 +114,18 @@ PATHS = [("staged", B.KV_PATH_STAGED), ("zerocopy", B.KV_PATH_ZEROCOPY), ("ce2d"
          ("naive", B.KV_PATH_NAIVE), ("auto", B.KV_PATH_AUTO)]
 
 
-def paths(out, max_payload_gb: float, device_layout: int = 0) -> None:
+def paths(out, max_payload_gb: float, device_layout: int = 0, kv_heads: int = 8) -> None:
     import torch
     rows = []
     payloads = [p for p in (64e6, 256e6, 1e9, 4e9, 8e9) if p <= max_payload_gb * 1e9 + 1]
     for bs in (8, 16, 32, 64):
         for contiguous in (True, False):
             for payload in payloads:
-                shape = W.KVShape(32, bs)
+                shape = W.KVShape(32, bs, kv_heads)
                 n = max(1, int(payload // shape.block_bytes))
                 # random tables: a host pool much larger than the payload, so that ids are truly scattered
                 nb_host = 2 * n + 16 if contiguous else int(min(16 * n, 40e9 // shape.block_bytes))
-                w = W.config4_sweep_case(bs, contiguous, payload, nb_host=max(nb_host, 2 * n + 16))
+                w = W.config4_sweep_case(bs, contiguous, payload, nb_host=max(nb_host, 2 * n + 16), kv_heads=kv_heads)
                 rot = w.steps[0]
                 dev = torch.empty(w.nb_gpu * shape.block_bytes, dtype=torch.uint8, device="cuda:0")
                 probe_bi = B.kv_probe_link(0, 256 * M, 2)["bi_sum_gbs"]
@@ -546,6 +546,8 @@ def main() -> None:
     ap.add_argument("--block-size", type=int, default=16, help="latency: tokens per block (8 = 1 MiB blocks, 16 = 2 MiB, 32 = 4 MiB)")
     ap.add_argument("--device-layout", choices=["layer-first", "block-first"], default="layer-first",
                     help="paths: device pool layout (block-first = the paper's redesigned storage order)")
+    ap.add_argument("--kv-heads", type=int, default=8,
+                    help="paths: KV heads held by this GPU (8 = the whole 8B shape; 1, 2 or 4 = one rank's shard under tensor parallelism)")
     a = ap.parse_args()
     import torch
     if not torch.cuda.is_available():
@@ -554,7 +556,7 @@ def main() -> None:
     if a.what == "probe":
         probe(out)
     elif a.what == "paths":
-        paths(out, a.max_payload_gb, 1 if a.device_layout == "block-first" else 0)
+        paths(out, a.max_payload_gb, 1 if a.device_layout == "block-first" else 0, a.kv_heads)
     elif a.what == "overlap":
         overlap(out)
     elif a.what == "latency":

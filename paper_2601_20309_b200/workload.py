@@ -454,11 +454,12 @@ def config3_70b(seed: int = MASTER_SEED + 3, nb_gpu: Optional[int] = None, nb_ho
 
 def config4_sweep_case(block_size: int, contiguous: bool, payload_bytes: float,
                        seed: int = MASTER_SEED + 4, nb_gpu: Optional[int] = None,
-                       nb_host: Optional[int] = None, num_layers: int = 32) -> Workload:
+                       nb_host: Optional[int] = None, num_layers: int = 32, kv_heads: int = 8) -> Workload:
     """One cell of the block-size / fragmentation sweep on the 8B shape: ``payload_bytes`` per
-    direction, block tables either ascending runs of ids or a uniformly random permutation."""
+    direction, block tables either ascending runs of ids or a uniformly random permutation.
+    ``kv_heads`` below 8 gives the shard one rank of a tensor-parallel group would hold."""
     rng = np.random.default_rng(seed + block_size + (0 if contiguous else 1000))
-    shape = KVShape(num_layers, block_size)
+    shape = KVShape(num_layers, block_size, kv_heads)
     n = max(1, int(payload_bytes // shape.block_bytes))
     nb_gpu = 2 * n + 16 if nb_gpu is None else nb_gpu
     nb_host = 2 * n + 16 if nb_host is None else nb_host

@@ -616,3 +616,48 @@ def test_random_shapes_lists_and_staging_sizes(seed):
         assert p.pool.kv_get_stats()["device_status"] == 0
     finally:
         p.close()
+
+
+# segment bytes -> (block_size, kv_heads, head_dim): every ring shape of the bulk kernel, from one issuing
+# warp with 16 KiB stages down to sixteen warps with 1 KiB stages, plus sizes between the powers of two
+SMALL_SEGMENTS = {512: (4, 1, 64), 1024: (8, 1, 64), 1536: (4, 3, 64), 2048: (8, 1, 128), 4096: (16, 1, 128),
+                  6144: (8, 3, 128), 8192: (16, 2, 128), 12288: (16, 3, 128), 16384: (16, 4, 128),
+                  20480: (16, 5, 128)}
+
+
+@pytest.mark.parametrize("path", [1, 2], ids=["zerocopy", "staged"])
+@pytest.mark.parametrize("seg", sorted(SMALL_SEGMENTS))
+def test_small_segments_take_every_ring_shape(seg, path):
+    """Shards of a tensor-parallel group and small block sizes have small segments, which the bulk kernel
+    moves with several issuing warps per CTA: lists long and short (fewer items than warps in some CTAs),
+    gather and scatter on their own, rotations on both paths, all against the oracle."""
+    bs, kv, hd = SMALL_SEGMENTS[seg]
+    shape = W.KVShape(3, bs, kv, hd)
+    assert shape.words_per_plane * 2 == seg
+    nbg, nbh = 700, 900
+    p = _pair(shape, nbg, nbh, seed=seg, path=path)
+    try:
+        import torch
+        rng = np.random.default_rng(seg + path)
+        for n in (1, 3, 37, 300):
+            og = rng.choice(nbg, n, replace=False).astype(np.int32)
+            oh = rng.choice(nbh, n, replace=False).astype(np.int32)
+            ig = rng.choice(np.setdiff1d(np.arange(nbg), og), n, replace=False).astype(np.int32)
+            ih = rng.choice(np.setdiff1d(np.arange(nbh), oh), n, replace=False).astype(np.int32)
+            assert p.rotate_both(W.Rotation(og, oh, ih, ig, np.zeros(1), np.zeros(1))) == 0
+            p.assert_equal(f"segment {seg}, path {path}, rotate of {n}")
+            # the device leg alone: gather into a buffer, scatter it to other blocks
+            buf = torch.zeros(n * shape.block_bytes, dtype=torch.uint8, device="cuda:0")
+            assert p.pool.kv_gather_blocks(og, buf.data_ptr()) == 0
+            p.pool.kv_sync()
+            want = np.concatenate([p.oracle.g_block(int(b)) for b in og])
+            assert np.array_equal(buf.cpu().numpy(), want), (seg, n)
+            assert p.pool.kv_scatter_blocks(buf.data_ptr(), ig) == 0
+            for s_, d_ in zip(og, ig):                      # the model's side of it: plane by plane
+                for l in range(shape.num_layers):
+                    for plane in range(2):
+                        p.oracle.g_seg(l, plane, int(d_))[:] = p.oracle.g_seg(l, plane, int(s_))
+            p.assert_equal(f"segment {seg}, path {path}, scatter of {n}")
+        assert p.pool.kv_get_stats()["device_status"] == 0
+    finally:
+        p.close()
