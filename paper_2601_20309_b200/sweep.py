@@ -11,6 +11,14 @@
         contiguous or uniformly random, payload 64 MB .. G GB per direction, each direction alone
         and both at once, on every transfer path.  Its result is the table behind kv_path_for.
 
+    python -m paper_2601_20309_b200.sweep paths --kv-heads H ...
+        The same sweep for the shard one rank of a tensor-parallel group holds (H = 4, 2 or 1 of the 8 KV
+        heads): segments and blocks shrink by 8 / H.
+
+    python -m paper_2601_20309_b200.sweep segments [--out FILE]
+        Rates against segment size, 32 KiB (the 8B shape) down to 1 KiB (small shards): gather and scatter
+        of 2 GiB of scattered blocks HBM to HBM, and the zero-copy kernels over the link, 512 MiB each way.
+
     python -m paper_2601_20309_b200.sweep overlap [--out FILE]
         Rotation beside compute (the paper's cross-iteration pipeline, section 4.3.2, hides transfers
         behind model execution): a rotation of 2 GiB each way runs while a stand-in for a decode step
@@ -168,6 +176,53 @@ def paths(out, max_payload_gb: float, device_layout: int = 0, kv_heads: int = 8)
         f = lambda k: "%s / %s / %s" % (r[k]["out"], r[k]["in"], r[k]["both"]) if k in r else "-"
         print(f"| {r['block_size']} | {r['blk_mib']:g} | {r['tables']} | {r['payload_mb']} | {r['probe_bi_gbs']} | "
               f"{f('staged')} | {f('zerocopy')} | {f('ce2d')} | {f('naive')} | {f('auto')} | {r['auto_took']} |")
+
+
+def segments(out) -> None:
+    """Rates against segment size: the device leg (gather / scatter of 2 GiB of scattered blocks, HBM to
+    HBM) and the zero-copy kernels (512 MiB each way over the link), for the 8B shape and the shards of it
+    that one rank of a tensor-parallel group holds, down to 1 KiB segments."""
+    import numpy as np
+    import torch
+    rows = []
+    for kv, bs, hd in ((8, 16, 128), (4, 16, 128), (2, 16, 128), (1, 32, 128), (1, 16, 128), (1, 8, 128), (1, 8, 64)):
+        shape = W.KVShape(32, bs, kv, hd)
+        blk = shape.block_bytes
+        nbg, nbh = 4 * G // blk - 37, 2 * G // blk
+        n = nbg // 2
+        dev = torch.empty(nbg * blk, dtype=torch.uint8, device="cuda:0")
+        stage = torch.empty(n * blk, dtype=torch.uint8, device="cuda:0")
+        pool = B.KVPool(shape.num_layers, bs, kv, hd, nbg, nbh, dev.data_ptr(), path=B.KV_PATH_ZEROCOPY)
+        rng = np.random.default_rng(3)
+        gp, hp = rng.permutation(nbg).astype(np.int32), rng.permutation(nbh).astype(np.int32)
+        ids = gp[:n]
+
+        def mean_ms(fn, reps=7, skip=3):
+            ts = []
+            for _ in range(reps):
+                fn()
+                pool.kv_sync()
+                ts.append(pool.kv_get_stats()["last_union_ms"])
+            return float(np.mean(ts[skip:]))
+
+        rec = {"kv_heads": kv, "block_size": bs, "head_dim": hd, "seg_kib": shape.words_per_plane * 2 / K,
+               "blk_kib": blk / K, "blocks_gathered": int(n),
+               "gather_tbs": round(2.0 * n * blk / mean_ms(lambda: pool.kv_gather_blocks(ids, stage.data_ptr())) / 1e9, 3),
+               "scatter_tbs": round(2.0 * n * blk / mean_ms(lambda: pool.kv_scatter_blocks(stage.data_ptr(), ids)) / 1e9, 3)}
+        m = (512 * M) // blk
+        og, ig, oh, ih = gp[:m], gp[m:2 * m], hp[:m], hp[m:2 * m]
+        rec["zerocopy_out_gbs"] = round(m * blk / mean_ms(lambda: pool.kv_swap_out(og, oh), 4, 1) / 1e6, 1)
+        rec["zerocopy_in_gbs"] = round(m * blk / mean_ms(lambda: pool.kv_swap_in(ih, ig), 4, 1) / 1e6, 1)
+        rec["zerocopy_both_gbs"] = round(2 * m * blk / mean_ms(lambda: pool.kv_rotate(og, oh, ih, ig), 4, 1) / 1e6, 1)
+        pool.destroy()
+        del dev, stage
+        torch.cuda.empty_cache()
+        rows.append(rec)
+        _emit(rec, out)
+    print("\n| KV heads | block | head dim | SEG KiB | BLK KiB | gather TB/s | scatter TB/s | zero-copy out / in / both GB/s |\n|---|---|---|---|---|---|---|---|")
+    for r in rows:
+        print(f"| {r['kv_heads']} | {r['block_size']} | {r['head_dim']} | {r['seg_kib']:g} | {r['blk_kib']:g} | {r['gather_tbs']} | "
+              f"{r['scatter_tbs']} | {r['zerocopy_out_gbs']} / {r['zerocopy_in_gbs']} / {r['zerocopy_both_gbs']} |")
 
 
 def overlap(out) -> None:
@@ -537,7 +592,7 @@ def budget(out, b_xfer: int) -> None:
 
 def main() -> None:
     ap = argparse.ArgumentParser()
-    ap.add_argument("what", choices=["probe", "paths", "overlap", "latency", "budget", "handoff", "lvf", "lvf-table"])
+    ap.add_argument("what", choices=["probe", "paths", "segments", "overlap", "latency", "budget", "handoff", "lvf", "lvf-table"])
     ap.add_argument("--eager-blocks", type=int, default=0, help="lvf-table: full blocks copied out in the background per step")
     ap.add_argument("--steps", type=int, default=300, help="lvf: steps to time")
     ap.add_argument("--out", default=None)
@@ -557,6 +612,8 @@ def main() -> None:
         probe(out)
     elif a.what == "paths":
         paths(out, a.max_payload_gb, 1 if a.device_layout == "block-first" else 0, a.kv_heads)
+    elif a.what == "segments":
+        segments(out)
     elif a.what == "overlap":
         overlap(out)
     elif a.what == "latency":
