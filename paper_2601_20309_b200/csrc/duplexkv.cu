@@ -2022,7 +2022,7 @@ extern "C" int32_t kv_gather_blocks_static(const void *device_base, int32_t num_
         // once per device, with that device current
         void *ptr = nullptr;
         KV_CUDA(nullptr, cudaGetSymbolAddress((void **)&ptr, kv_static_scratch));
-        KV_CUDA(nullptr, BulkHbm::prepare());
+        KV_CUDA(nullptr, prepare_bulk_kernels());
         g_static_scratch[dev] = ptr;
     }
     int2 *pairs = (int2 *)g_static_scratch[dev];
@@ -2053,7 +2053,7 @@ extern "C" int32_t kv_gather_blocks_static(const void *device_base, int32_t num_
     kd.src_blocks = (int)num_gpu_blocks;
     kd.dst_blocks = (int)n;
     kd.ctas = clamp_ctas(job, kd, sm_count > 0 ? sm_count : 1);
-    BulkHbm::launch(kd.ctas, st, job);
+    launch_bulk(nullptr, job, kd.ctas, st, false);
     KV_CUDA(nullptr, cudaGetLastError());
     unsigned int seen = 0;
     KV_CUDA(nullptr, cudaMemcpyAsync(&seen, status, sizeof(seen), cudaMemcpyDeviceToHost, st));
