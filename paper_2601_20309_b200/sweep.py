@@ -15,9 +15,10 @@
         The same sweep for the shard one rank of a tensor-parallel group holds (H = 4, 2 or 1 of the 8 KV
         heads): segments and blocks shrink by 8 / H.
 
-    python -m paper_2601_20309_b200.sweep segments [--out FILE]
+    python -m paper_2601_20309_b200.sweep segments [--pool-gib P] [--out FILE]
         Rates against segment size, 32 KiB (the 8B shape) down to 1 KiB (small shards): gather and scatter
-        of 2 GiB of scattered blocks HBM to HBM, and the zero-copy kernels over the link, 512 MiB each way.
+        of half of a P GiB pool's blocks (P = 4: 2 GiB), scattered, HBM to HBM, and the zero-copy kernels over
+        the link, P/8 GiB each way.
 
     python -m paper_2601_20309_b200.sweep overlap [--out FILE]
         Rotation beside compute (the paper's cross-iteration pipeline, section 4.3.2, hides transfers
@@ -178,9 +179,9 @@ def paths(out, max_payload_gb: float, device_layout: int = 0, kv_heads: int = 8)
               f"{f('staged')} | {f('zerocopy')} | {f('ce2d')} | {f('naive')} | {f('auto')} | {r['auto_took']} |")
 
 
-def segments(out) -> None:
+def segments(out, pool_gib: int = 4) -> None:
     """Rates against segment size: the device leg (gather / scatter of 2 GiB of scattered blocks, HBM to
-    HBM) and the zero-copy kernels (512 MiB each way over the link), for the 8B shape and the shards of it
+    HBM) and the zero-copy kernels (an eighth of the pool size each way over the link), for the 8B shape and the shards of it
     that one rank of a tensor-parallel group holds, down to 1 KiB segments."""
     import numpy as np
     import torch
@@ -188,7 +189,7 @@ def segments(out) -> None:
     for kv, bs, hd in ((8, 16, 128), (4, 16, 128), (2, 16, 128), (1, 32, 128), (1, 16, 128), (1, 8, 128), (1, 8, 64)):
         shape = W.KVShape(32, bs, kv, hd)
         blk = shape.block_bytes
-        nbg, nbh = 4 * G // blk - 37, 2 * G // blk
+        nbg, nbh = pool_gib * G // blk - 37, pool_gib * G // 2 // blk
         n = nbg // 2
         dev = torch.empty(nbg * blk, dtype=torch.uint8, device="cuda:0")
         stage = torch.empty(n * blk, dtype=torch.uint8, device="cuda:0")
@@ -209,7 +210,7 @@ def segments(out) -> None:
                "blk_kib": blk / K, "blocks_gathered": int(n),
                "gather_tbs": round(2.0 * n * blk / mean_ms(lambda: pool.kv_gather_blocks(ids, stage.data_ptr())) / 1e9, 3),
                "scatter_tbs": round(2.0 * n * blk / mean_ms(lambda: pool.kv_scatter_blocks(stage.data_ptr(), ids)) / 1e9, 3)}
-        m = (512 * M) // blk
+        m = (pool_gib * 128 * M) // blk
         og, ig, oh, ih = gp[:m], gp[m:2 * m], hp[:m], hp[m:2 * m]
         rec["zerocopy_out_gbs"] = round(m * blk / mean_ms(lambda: pool.kv_swap_out(og, oh), 4, 1) / 1e6, 1)
         rec["zerocopy_in_gbs"] = round(m * blk / mean_ms(lambda: pool.kv_swap_in(ih, ig), 4, 1) / 1e6, 1)
@@ -601,6 +602,7 @@ def main() -> None:
     ap.add_argument("--block-size", type=int, default=16, help="latency: tokens per block (8 = 1 MiB blocks, 16 = 2 MiB, 32 = 4 MiB)")
     ap.add_argument("--device-layout", choices=["layer-first", "block-first"], default="layer-first",
                     help="paths: device pool layout (block-first = the paper's redesigned storage order)")
+    ap.add_argument("--pool-gib", type=int, default=4, help="segments: device pool size in GiB")
     ap.add_argument("--kv-heads", type=int, default=8,
                     help="paths: KV heads held by this GPU (8 = the whole 8B shape; 1, 2 or 4 = one rank's shard under tensor parallelism)")
     a = ap.parse_args()
@@ -613,7 +615,7 @@ def main() -> None:
     elif a.what == "paths":
         paths(out, a.max_payload_gb, 1 if a.device_layout == "block-first" else 0, a.kv_heads)
     elif a.what == "segments":
-        segments(out)
+        segments(out, a.pool_gib)
     elif a.what == "overlap":
         overlap(out)
     elif a.what == "latency":
