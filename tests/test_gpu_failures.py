@@ -64,6 +64,34 @@ def test_a_wait_that_runs_out_is_reported_and_the_device_stays_usable(path):
         q.close()
 
 
+@pytest.mark.parametrize("path", ["zerocopy", "staged"])
+def test_a_wait_that_runs_out_with_several_issuing_warps_per_cta(path):
+    """The same with 2 KiB segments, where every CTA runs several rings (one per warp): each ring's thread
+    records the timeout, waits for its own loads in flight and returns."""
+    shape = W.KVShape(2, 8, 1, 128)
+    nbg, nbh, n = 256, 512, 40
+    rng = np.random.default_rng(11)
+    pg, ph = rng.permutation(nbg).astype(np.int32), rng.permutation(nbh).astype(np.int32)
+    r = W.Rotation(pg[:n], ph[:n], ph[n:2 * n], pg[n:2 * n], np.zeros(1), np.zeros(1))
+    pid = {"zerocopy": 1, "staged": 2}[path]
+    p = _pair(shape, nbg, nbh, seed=5, path=pid)
+    try:
+        assert p.pool.kv_pool_set_wait_limit(0, 0) == 0
+        assert p.pool.kv_rotate(r.out_gpu, r.out_host, r.in_host, r.in_gpu, check=False) == 0
+        assert p.pool.kv_sync(check=False) == B.KV_ERR_TIMEOUT
+        assert p.pool.kv_get_stats()["device_status"] & 1
+        assert _guards_intact(p)
+    finally:
+        p.close()
+    q = _pair(shape, nbg, nbh, seed=5, path=pid)
+    try:
+        assert q.rotate_both(r) == 0
+        q.assert_equal("rotation on a fresh pool after the timed-out one")
+        assert q.pool.kv_get_stats()["device_status"] == 0
+    finally:
+        q.close()
+
+
 def test_wait_limit_arguments():
     w = W.config1_tiny()
     p = _pair(w.shape, w.nb_gpu, w.nb_host, seed=w.seed, path=1)
