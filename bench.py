@@ -499,9 +499,31 @@ def run_ours(args, rank: int, local_rank: int, world: int) -> None:
             except (MemoryError, B.KVError) as e:
                 cfg3 = {"skipped": f"not run on this box: {e}"}
 
+            # ---- the device leg against segment size: the 8B shape whole and as the shard one rank holds at
+            #      tensor-parallel degree 4 and 8 (block 16 and 8), 4 GiB pools, half of the blocks gathered
+            by_seg = []
+            for kv_h, bs_h, hd_h in ((8, 16, 128), (2, 16, 128), (1, 16, 128), (1, 8, 128), (1, 8, 64)):
+                sh = W.KVShape(shape.num_layers, bs_h, kv_h, hd_h)
+                nb_s = ((1 if args.small else 4) << 30) // sh.block_bytes - 37
+                ids_s = np.random.default_rng(3).permutation(nb_s)[:nb_s // 2].astype(np.int32)
+                dev_s = torch.empty(nb_s * sh.block_bytes, dtype=torch.uint8, device=dev)
+                out_s = torch.empty(len(ids_s) * sh.block_bytes, dtype=torch.uint8, device=dev)
+                pool_s = B.KVPool(sh.num_layers, bs_h, kv_h, hd_h, nb_s, 16, dev_s.data_ptr(), device_id=local_rank)
+                ts = []
+                for _ in range(8):
+                    pool_s.kv_gather_blocks(ids_s, out_s.data_ptr())
+                    pool_s.kv_sync()
+                    ts.append(pool_s.kv_get_stats()["last_union_ms"])
+                pool_s.destroy()
+                g_s = M.gbs(2.0 * len(ids_s) * sh.block_bytes, float(np.mean(ts[3:])))
+                by_seg.append({"kv_heads": kv_h, "block_size": bs_h, "head_dim": hd_h, "segment_bytes": sh.words_per_plane * 2,
+                               "gather_gbs": g_s, "frac_of_measured_hbm": g_s / peaks["hbm_gbs"]})
+                del dev_s, out_s
+
         extra = {"paths": paths, "singles": singles, "lat_us": lat_us, "lat_blocks": lat_blocks, "leg": leg,
                  "leg_bytes": leg_bytes, "probe2": probe2, "contiguous_host": contiguous_host, "table": tb,
-                 "lat_paths": lat_paths, "one_us": one_us, "table1": table1, "cfg5": cfg5, "cfg3": cfg3}
+                 "lat_paths": lat_paths, "one_us": one_us, "table1": table1, "cfg5": cfg5, "cfg3": cfg3,
+                 "by_seg": by_seg if not args.quick else None}
 
     pool.destroy()
     del device_pool
@@ -599,6 +621,7 @@ def run_ours(args, rank: int, local_rank: int, world: int) -> None:
             "config3": extra["cfg3"],
             "config4_table1": extra["table1"],
             "config5": extra["cfg5"],
+            "device_leg_by_segment": extra["by_seg"],
             "cpu_baseline": {"value": cpu_val, "unit": UNIT, "cores": threads, "kind": "oracle", "sample": sample,
                              "single_thread_value": cpu_1},
         }
