@@ -225,10 +225,16 @@ bool ldst32(const kv_pool *p, bool link)
 void fill_geometry(const kv_pool *p, KvJob &job, bool link = false)
 {
     const int max_chunk = use_ldst(p) ? LDST_CHUNK : (link ? link_stage(p) : BULK_STAGE);
-    job.planes = p->planes;
-    job.seg = (int)p->seg;
-    job.chunk = (int)std::min<int64_t>(p->seg, max_chunk);
-    job.cps = (int)((p->seg + job.chunk - 1) / job.chunk);
+    // With a block-first device pool against staging, a packed buffer or a block-first host pool, both
+    // sides hold a block's planes back to back: the block is one run of BLK bytes and is moved as such,
+    // however small its segments are.
+    const bool whole_blocks = dev_block_first(p) && (!link || p->cfg.host_layout == KV_HOST_BLOCK_FIRST) &&
+                              p->blk <= (int64_t)INT32_MAX;
+    const int64_t run = whole_blocks ? p->blk : p->seg;
+    job.planes = whole_blocks ? 1 : p->planes;
+    job.seg = (int)run;
+    job.chunk = (int)std::min<int64_t>(run, max_chunk);
+    job.cps = (int)((run + job.chunk - 1) / job.chunk);
     job.status = p->status_dev;
     job.wait_polls = p->wait_polls;
     job.wait_ns = p->wait_ns;

@@ -625,17 +625,19 @@ SMALL_SEGMENTS = {512: (4, 1, 64), 1024: (8, 1, 64), 1536: (4, 3, 64), 2048: (8,
                   20480: (16, 5, 128)}
 
 
+@pytest.mark.parametrize("device_layout", [0, 1], ids=["devlayerfirst", "devblockfirst"])
 @pytest.mark.parametrize("path", [1, 2], ids=["zerocopy", "staged"])
 @pytest.mark.parametrize("seg", sorted(SMALL_SEGMENTS))
-def test_small_segments_take_every_ring_shape(seg, path):
+def test_small_segments_take_every_ring_shape(seg, path, device_layout):
     """Shards of a tensor-parallel group and small block sizes have small segments, which the bulk kernel
     moves with several issuing warps per CTA: lists long and short (fewer items than warps in some CTAs),
-    gather and scatter on their own, rotations on both paths, all against the oracle."""
+    gather and scatter on their own, rotations on both paths, all against the oracle.  With a block-first
+    device pool the same blocks travel as whole runs of BLK bytes."""
     bs, kv, hd = SMALL_SEGMENTS[seg]
     shape = W.KVShape(3, bs, kv, hd)
     assert shape.words_per_plane * 2 == seg
     nbg, nbh = 700, 900
-    p = _pair(shape, nbg, nbh, seed=seg, path=path)
+    p = _pair(shape, nbg, nbh, seed=seg, path=path, device_layout=device_layout)
     try:
         import torch
         rng = np.random.default_rng(seg + path)
