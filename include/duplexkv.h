@@ -397,6 +397,16 @@ int32_t kv_completion_event(kv_pool_t *pool, int32_t direction, void **event);
  * 64).  How many SMs a rotation may occupy beside model execution is a sizing decision of the caller. */
 int32_t kv_pool_set_ctas(kv_pool_t *pool, int32_t ctas_out, int32_t ctas_in);
 
+/* Which shape of the bulk-copy kernel a launch takes for segments of segment_bytes (host logic, no device
+ * needed): the bytes of one work item, and the ring each issuing warp runs -- stage size, stages, loads
+ * ahead of the stores -- and the issuing warps per CTA.  over_link = 0: HBM to HBM (pack, unpack, gather,
+ * scatter); 1: the zero-copy kernels, with the pool's link_variant.  An item never exceeds a stage, and a
+ * CTA uses stage_bytes * stages * warps bytes of dynamic shared memory (at most 227 KiB).  Any out pointer
+ * may be NULL.  KV_ERR_INVALID_ARG for a segment size that is not a positive multiple of 16 or an unknown
+ * variant. */
+int32_t kv_debug_ring_shape(int64_t segment_bytes, int32_t over_link, int32_t link_variant, int32_t *item_bytes,
+                            int32_t *stage_bytes, int32_t *stages, int32_t *ahead, int32_t *warps);
+
 /* The predicate behind KV_FLAG_DEBUG_BOUNDS as a host function: 1 when both ids lie inside their pools. */
 int32_t kv_debug_pair_in_bounds(int32_t src_id, int32_t dst_id, int32_t src_blocks, int32_t dst_blocks);
 

@@ -110,7 +110,7 @@ EXPORTS = ["kv_pool_create", "kv_pool_destroy", "kv_pool_set_path", "kv_swap_out
            "kv_req_append", "kv_eager_rotate", "kv_req_rotate", "kv_req_preempt", "kv_req_resume", "kv_req_finish",
            "kv_req_info", "kv_req_blocks", "kv_table_get_stats", "kv_table_fail_pool_call",
            "kv_pool_set_wait_limit", "kv_pool_set_call_timing", "kv_completion_event", "kv_pool_set_ctas",
-           "kv_debug_pair_in_bounds", "kv_rotate_req"]
+           "kv_debug_pair_in_bounds", "kv_rotate_req", "kv_debug_ring_shape"]
 
 _lib = None
 
@@ -195,6 +195,8 @@ def lib() -> C.CDLL:
     L.kv_pool_set_ctas.argtypes = [vp, C.c_int32, C.c_int32]
     L.kv_debug_pair_in_bounds.restype = C.c_int32
     L.kv_debug_pair_in_bounds.argtypes = [C.c_int32] * 4
+    L.kv_debug_ring_shape.restype = C.c_int32
+    L.kv_debug_ring_shape.argtypes = [C.c_int64, C.c_int32, C.c_int32] + [C.POINTER(C.c_int32)] * 5
     L.kv_rotate_req.restype = C.c_int32
     L.kv_rotate_req.argtypes = [vp, i32p, i32p, i64, C.POINTER(C.c_int64), i64, i32p, i32p, i64, C.POINTER(C.c_int64), i64]
     L.kv_pool_set_call_timing.restype = C.c_int32
@@ -232,6 +234,15 @@ def kv_seg_bytes(block_size: int, kv_heads: int, head_dim: int) -> int:
 
 def kv_blk_bytes(num_layers: int, block_size: int, kv_heads: int, head_dim: int) -> int:
     return lib().kv_blk_bytes(num_layers, block_size, kv_heads, head_dim)
+
+
+def kv_debug_ring_shape(segment_bytes: int, over_link: bool = False, link_variant: int = 0, check: bool = True):
+    """(rc, dict): item bytes, stage bytes, stages, loads ahead and issuing warps of the bulk kernel for this segment size."""
+    v = [C.c_int32() for _ in range(5)]
+    rc = lib().kv_debug_ring_shape(segment_bytes, int(over_link), link_variant, *[C.byref(x) for x in v])
+    if check and rc != KV_OK:
+        raise KVError(rc, lib().kv_last_error(None).decode())
+    return rc, dict(zip(("item_bytes", "stage_bytes", "stages", "ahead", "warps"), (x.value for x in v)))
 
 
 def kv_debug_pair_in_bounds(src_id: int, dst_id: int, src_blocks: int, dst_blocks: int) -> bool:

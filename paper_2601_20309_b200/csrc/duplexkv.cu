@@ -262,48 +262,59 @@ struct Bulk {
         kv_copy_bulk<STAGE, NS, AHEAD><<<grid, 32 * WARPS, smem, stream>>>(job);
     }
 };
-using BulkHbm = Bulk<BULK_STAGE, BULK_NS, BULK_AHEAD, 1>;
-using BulkHbm8k = Bulk<8192, SMALL_NS, SMALL_AHEAD, 2>;
-using BulkHbm4k = Bulk<4096, SMALL_NS, SMALL_AHEAD, 4>;
-using BulkHbm2k = Bulk<2048, SMALL_NS, SMALL_AHEAD, 8>;
-using BulkHbm1k = Bulk<1024, TINY_NS, TINY_AHEAD, 16>;
-using BulkLink = Bulk<LINK_STAGE, LINK_NS, LINK_AHEAD, 1>;
-using BulkLink1 = Bulk<LINK1_STAGE, LINK1_NS, LINK1_AHEAD, 1>;
-using BulkLink2 = Bulk<LINK2_STAGE, LINK2_NS, LINK2_AHEAD, 1>;
-using BulkLink4k = Bulk<4096, SMALL_LINK_NS, SMALL_LINK_AHEAD, 2>;
-using BulkLink2k = Bulk<2048, SMALL_LINK_NS, SMALL_LINK_AHEAD, 4>;
-using BulkLink1k = Bulk<1024, SMALL_LINK_NS, SMALL_LINK_AHEAD, 8>;
+// every shape of the bulk kernel that a launch can take, in one table: geometry, and how to prepare and launch it
+struct BulkShape {
+    int stage, stages, ahead, warps;
+    cudaError_t (*prepare)();
+    void (*launch)(int grid, cudaStream_t stream, const KvJob &job);
+};
+template <typename B, int STAGE, int NS, int AHEAD, int WARPS>
+constexpr BulkShape bulk_shape()
+{
+    return BulkShape{STAGE, NS, AHEAD, WARPS, B::prepare, B::launch};
+}
+#define KV_BULK_SHAPE(STAGE, NS, AHEAD, WARPS) bulk_shape<Bulk<STAGE, NS, AHEAD, WARPS>, STAGE, NS, AHEAD, WARPS>()
+const BulkShape g_bulk_shapes[] = {
+    /* 0..4: HBM to HBM, by item size */
+    KV_BULK_SHAPE(BULK_STAGE, BULK_NS, BULK_AHEAD, 1), KV_BULK_SHAPE(8192, SMALL_NS, SMALL_AHEAD, 2),
+    KV_BULK_SHAPE(4096, SMALL_NS, SMALL_AHEAD, 4),     KV_BULK_SHAPE(2048, SMALL_NS, SMALL_AHEAD, 8),
+    KV_BULK_SHAPE(1024, TINY_NS, TINY_AHEAD, 16),
+    /* 5..7: over the link, link_variant 0 / 1 / 2 */
+    KV_BULK_SHAPE(LINK_STAGE, LINK_NS, LINK_AHEAD, 1), KV_BULK_SHAPE(LINK1_STAGE, LINK1_NS, LINK1_AHEAD, 1),
+    KV_BULK_SHAPE(LINK2_STAGE, LINK2_NS, LINK2_AHEAD, 1),
+    /* 8..10: over the link, small items */
+    KV_BULK_SHAPE(4096, SMALL_LINK_NS, SMALL_LINK_AHEAD, 2), KV_BULK_SHAPE(2048, SMALL_LINK_NS, SMALL_LINK_AHEAD, 4),
+    KV_BULK_SHAPE(1024, SMALL_LINK_NS, SMALL_LINK_AHEAD, 8)};
+#undef KV_BULK_SHAPE
 
 cudaError_t prepare_bulk_kernels()
 {
-    cudaError_t (*const all[])() = {BulkHbm::prepare,   BulkHbm8k::prepare,  BulkHbm4k::prepare,  BulkHbm2k::prepare,
-                                    BulkHbm1k::prepare, BulkLink::prepare,   BulkLink1::prepare,  BulkLink2::prepare,
-                                    BulkLink4k::prepare, BulkLink2k::prepare, BulkLink1k::prepare};
-    for (auto fn : all) {
-        const cudaError_t rc = fn();
+    for (const BulkShape &b : g_bulk_shapes) {
+        const cudaError_t rc = b.prepare();
         if (rc != cudaSuccess) return rc;
     }
     return cudaSuccess;
 }
 
-// the bulk kernel's shape for items of job.chunk bytes
+// the bulk kernel's shape for items of `chunk` bytes (never smaller than an item: a stage holds one)
+const BulkShape &bulk_shape_for(int chunk, bool link, int link_variant)
+{
+    if (link) {
+        if (chunk <= 1024) return g_bulk_shapes[10];
+        if (chunk <= 2048) return g_bulk_shapes[9];
+        if (chunk <= 4096) return g_bulk_shapes[8];
+        return g_bulk_shapes[link_variant == 1 ? 6 : (link_variant == 2 ? 7 : 5)];
+    }
+    if (chunk <= 1024) return g_bulk_shapes[4];
+    if (chunk <= 2048) return g_bulk_shapes[3];
+    if (chunk <= 4096) return g_bulk_shapes[2];
+    if (chunk <= 8192) return g_bulk_shapes[1];
+    return g_bulk_shapes[0];
+}
+
 void launch_bulk(const kv_pool *p, const KvJob &job, int grid, cudaStream_t stream, bool link)
 {
-    const int c = job.chunk;
-    if (link) {
-        if (c <= 1024) BulkLink1k::launch(grid, stream, job);
-        else if (c <= 2048) BulkLink2k::launch(grid, stream, job);
-        else if (c <= 4096) BulkLink4k::launch(grid, stream, job);
-        else if (p->cfg.link_variant == 1) BulkLink1::launch(grid, stream, job);
-        else if (p->cfg.link_variant == 2) BulkLink2::launch(grid, stream, job);
-        else BulkLink::launch(grid, stream, job);
-    } else {
-        if (c <= 1024) BulkHbm1k::launch(grid, stream, job);
-        else if (c <= 2048) BulkHbm2k::launch(grid, stream, job);
-        else if (c <= 4096) BulkHbm4k::launch(grid, stream, job);
-        else if (c <= 8192) BulkHbm8k::launch(grid, stream, job);
-        else BulkHbm::launch(grid, stream, job);
-    }
+    bulk_shape_for(job.chunk, link, p ? p->cfg.link_variant : 0).launch(grid, stream, job);
 }
 
 cudaError_t launch_job(kv_pool *p, const KvJob &job, cudaStream_t stream, bool link = false)
@@ -1718,6 +1729,23 @@ int32_t kv_pool_set_ctas(kv_pool_t *p, int32_t ctas_out, int32_t ctas_in)
     p->cfg.ctas_in = ctas_in;
     p->dir[0].ctas = ctas_out > 0 ? ctas_out : 64;
     p->dir[1].ctas = ctas_in > 0 ? ctas_in : 64;
+    return KV_OK;
+}
+
+int32_t kv_debug_ring_shape(int64_t segment_bytes, int32_t over_link, int32_t link_variant, int32_t *item_bytes,
+                            int32_t *stage_bytes, int32_t *stages, int32_t *ahead, int32_t *warps)
+{
+    if (segment_bytes <= 0 || segment_bytes % 16 != 0 || link_variant < 0 || link_variant > 2)
+        return fail(nullptr, KV_ERR_INVALID_ARG, "segment_bytes must be a positive multiple of 16, link_variant 0..2");
+    // as fill_geometry and launch_bulk decide it
+    const int max_chunk = over_link ? (link_variant == 1 ? LINK1_STAGE : (link_variant == 2 ? LINK2_STAGE : LINK_STAGE)) : BULK_STAGE;
+    const int chunk = (int)std::min<int64_t>(segment_bytes, max_chunk);
+    const BulkShape &b = bulk_shape_for(chunk, over_link != 0, link_variant);
+    if (item_bytes) *item_bytes = chunk;
+    if (stage_bytes) *stage_bytes = b.stage;
+    if (stages) *stages = b.stages;
+    if (ahead) *ahead = b.ahead;
+    if (warps) *warps = b.warps;
     return KV_OK;
 }
 
