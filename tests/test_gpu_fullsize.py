@@ -194,3 +194,25 @@ def test_config4_sweep_cells_at_full_payload(bs, contiguous, payload):
         assert t.B.PATH_NAMES[t.pool.kv_get_stats()["last_path_out"]] == "staged"
     finally:
         t.close()
+
+
+@pytest.mark.parametrize("bs,kv_heads,contiguous,took", [(16, 1, False, "zerocopy"), (8, 1, True, "staged"), (32, 2, False, "staged")],
+                         ids=["tp8-block16-random", "tp8-block8-contiguous", "tp4-block32-random"])
+def test_tensor_parallel_shard_cells_at_full_payload(bs, kv_heads, contiguous, took):
+    """The shard one rank of a tensor-parallel group holds (1 or 2 of the 8 KV heads: 4 KiB, 2 KiB and 16 KiB
+    segments, 256 KiB, 128 KiB and 1 MiB blocks), 2 GB each way, default path: scattered small blocks through the
+    zero-copy kernels (several issuing warps per CTA), neighbouring ids and 1 MiB blocks staged."""
+    w = W.config4_sweep_case(bs, contiguous, 2e9, kv_heads=kv_heads)
+    t = _FullSize(w)
+    try:
+        r = w.steps[0]
+        t.swap_out(r.out_gpu, r.out_host)
+        moved = t.verify("swap-out alone", n_read_back=4)
+        assert moved == (0, r.n_out)
+        t.swap_in(r.in_host, r.in_gpu)
+        t.rotate(r)
+        moved = t.verify("swap-in alone, then both at once", n_read_back=4)
+        assert moved == (r.n_in, r.n_out)
+        assert t.B.PATH_NAMES[t.pool.kv_get_stats()["last_path_out"]] == took
+    finally:
+        t.close()
