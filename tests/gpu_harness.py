@@ -7,6 +7,11 @@ from paper_2601_20309_b200 import binding as B
 from paper_2601_20309_b200 import workload as W
 
 
+# initial content of the pools of the last Pair built (one entry): many tests start from the same pools, and
+# generating a block's content on the CPU is the slow part of building them
+_INITIAL = {}
+
+
 class Pair:
     """A GPU pool (through the C ABI) and the byte oracle holding the same logical content."""
 
@@ -19,18 +24,26 @@ class Pair:
                                  dev_layout=device_layout)
         o = self.oracle
         wpp = s.words_per_plane
-        G16 = o.G.view(np.uint16)
-        H16 = o.Hs.view(np.uint16)
-        for b in range(nb_gpu):
-            words = W.block_words(seed, W.POOL_GPU, b, s.words_per_block).reshape(2 * s.num_layers, wpp)
-            for pl in range(2 * s.num_layers):
-                off = o.dev_off(pl // 2, pl % 2, b) // 2
-                G16[off:off + wpp] = words[pl]
-        for h in range(nb_host):
-            words = W.block_words(seed, W.POOL_HOST, h, s.words_per_block).reshape(2 * s.num_layers, wpp)
-            for pl in range(2 * s.num_layers):
-                off = o.host_off(h, pl // 2, pl % 2) // 2
-                H16[off:off + wpp] = words[pl]
+        key = (s, nb_gpu, nb_host, seed, host_layout, device_layout)
+        if _INITIAL.get("key") == key:                      # the previous test started from the same pools
+            o.G[:] = _INITIAL["G"]
+            o.Hs[:] = _INITIAL["Hs"]
+        else:
+            G16 = o.G.view(np.uint16)
+            H16 = o.Hs.view(np.uint16)
+            for b in range(nb_gpu):
+                words = W.block_words(seed, W.POOL_GPU, b, s.words_per_block).reshape(2 * s.num_layers, wpp)
+                for pl in range(2 * s.num_layers):
+                    off = o.dev_off(pl // 2, pl % 2, b) // 2
+                    G16[off:off + wpp] = words[pl]
+            for h in range(nb_host):
+                words = W.block_words(seed, W.POOL_HOST, h, s.words_per_block).reshape(2 * s.num_layers, wpp)
+                for pl in range(2 * s.num_layers):
+                    off = o.host_off(h, pl // 2, pl % 2) // 2
+                    H16[off:off + wpp] = words[pl]
+            _INITIAL.clear()
+            if o.G.size + o.Hs.size <= (4 << 30):
+                _INITIAL.update(key=key, G=o.G.copy(), Hs=o.Hs.copy())
         # the device pool sits between two guard areas of one block each, which no call may touch
         self.guard = -(-max(256, s.block_bytes) // 256) * 256
         self.buf = torch.full((o.G.size + 2 * self.guard,), 0xC3, dtype=torch.uint8, device="cuda:0")

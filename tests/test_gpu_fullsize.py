@@ -33,6 +33,36 @@ def _fit_host_pool(shape, nb_host):
     return nb_host
 
 
+# Pinning 120 GB takes the better part of a minute, so the tests of this file share one page-locked area:
+# a keeper pool of small blocks owns it, and every test's pool is created over that memory (the library
+# takes memory that is page-locked already as it is).
+_KEEPER = {"pool": None, "dev": None, "bytes": 0}
+
+
+def _shared_host(nbytes):
+    import torch
+    from paper_2601_20309_b200 import binding as B
+    k = _KEEPER
+    if k["pool"] is not None and k["bytes"] < nbytes:
+        k["pool"].destroy()
+        k["pool"] = None
+    if k["pool"] is None:
+        shape = W.KVShape(1, 16, 8, 128)                      # 64 KiB blocks
+        nb = -(-nbytes // shape.block_bytes)
+        k["dev"] = torch.empty(8 * shape.block_bytes, dtype=torch.uint8, device="cuda:0")
+        k["pool"] = B.KVPool(shape.num_layers, shape.block_size, shape.kv_heads, shape.head_dim, 8, nb, k["dev"].data_ptr())
+        k["bytes"] = nb * shape.block_bytes
+    return k["pool"].kv_host_ptr()[0]
+
+
+@pytest.fixture(scope="module", autouse=True)
+def _release_shared_host():
+    yield
+    if _KEEPER["pool"] is not None:
+        _KEEPER["pool"].destroy()
+        _KEEPER["pool"], _KEEPER["dev"], _KEEPER["bytes"] = None, None, 0
+
+
 class _FullSize:
     def __init__(self, w):
         import torch
@@ -46,7 +76,8 @@ class _FullSize:
             pytest.skip("not enough free device memory for this pool")
         self.dev = torch.empty(w.nb_gpu * shape.block_bytes, dtype=torch.uint8, device="cuda:0")
         self.pool = B.KVPool(shape.num_layers, shape.block_size, shape.kv_heads, shape.head_dim, w.nb_gpu, w.nb_host,
-                             self.dev.data_ptr(), flags=B.KV_FLAG_TIME_KERNELS)
+                             self.dev.data_ptr(), host_base=_shared_host(w.nb_host * shape.block_bytes),
+                             flags=B.KV_FLAG_TIME_KERNELS)
         host_base, _ = self.pool.kv_host_ptr()
         self.lay_g = F.Layout.device(self.dev.data_ptr(), shape, w.nb_gpu)
         self.lay_h = F.Layout.host(host_base, shape, w.nb_host)
