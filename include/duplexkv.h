@@ -124,8 +124,10 @@ typedef struct {
                                reads layer-first pools only                                               */
     int32_t link_variant;   /* shape of the zero-copy kernels' transfers (a measurement knob; 0 is the default and
                                the quickest found): bulk kernel: 0 = 8 KiB copies, 8-stage ring; 1 = 32 KiB
-                               copies, 4 stages; 2 = 64 KiB copies, 3 stages.  With KV_FLAG_LDST_KERNEL:
-                               1 = 32-byte instead of 16-byte vectors per thread                          */
+                               copies, 4 stages; 2 = 64 KiB copies, 3 stages (segments of 4 KiB and less take
+                               rings of their own size on several warps whatever the variant, see
+                               kv_debug_ring_shape).  With KV_FLAG_LDST_KERNEL: 1 = 32-byte instead of
+                               16-byte vectors per thread                                                 */
 } kv_pool_config_t;
 
 typedef struct {
