@@ -268,8 +268,12 @@ def run_ours(args, rank: int, local_rank: int, world: int) -> None:
     og, oh, ih, ig = (np.ascontiguousarray(x, np.int32) for x in (rot.out_gpu, rot.out_host, rot.in_host, rot.in_gpu))
     args_raw = (ptr(og), ptr(oh), len(og), ptr(ih), ptr(ig), len(ig))
 
+    issue_s = []                        # host time inside kv_rotate (validation, planning, launches, transfers queued)
+
     def step():
+        t_call = time.perf_counter()
         rc = pool.kv_rotate_raw(*args_raw)
+        issue_s.append(time.perf_counter() - t_call)
         if rc != 0:
             raise RuntimeError(f"kv_rotate failed: {rc} {pool.kv_last_error()}")
         pool.kv_sync()
@@ -594,7 +598,8 @@ def run_ours(args, rank: int, local_rank: int, world: int) -> None:
                        "l2": "inputs larger than L2 (3.9 GB per direction per step)", "replicas": world,
                        "pin_seconds": round(pin_s, 1)},
             "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": bytes_in + 8 * (rot.n_out + rot.n_in),
-                    "d2h_bytes_per_step": bytes_out, "ms_per_step": wall_total_s * 1e3 / args.steps},
+                    "d2h_bytes_per_step": bytes_out, "ms_per_step": wall_total_s * 1e3 / args.steps,
+                    "host_ms_inside_kv_rotate": float(np.median(issue_s[-args.steps:])) * 1e3},
             "gpu_launches": int(launches), "ce_transfers": int(ce_copies),
             "overlap": overlap_of(windows),
             "clocks": clocks,
