@@ -93,7 +93,11 @@ typedef struct {
     void   *device_base;    /* DEVICE pointer, required: >= num_gpu_blocks*BLK bytes, 256-byte aligned;
                                borrowed (typically a torch tensor's storage)                              */
     void   *host_base;      /* HOST pointer or NULL.  NULL: the library allocates num_host_blocks*BLK
-                               bytes of mapped pinned memory and owns it.  Non-NULL: caller memory of that
+                               bytes of mapped pinned memory and owns it (an anonymous mapping that asks for
+                               transparent huge pages, touched by several threads and then registered with
+                               CUDA, which page-locks several times faster than cudaHostAlloc; cudaHostAlloc
+                               when that fails, when the box has less than that much memory available, or
+                               when the environment says DUPLEXKV_HOST_ALLOC=cuda).  Non-NULL: caller memory of that
                                size, 4096-byte aligned; the library page-locks it for the pool's lifetime.
                                Memory that is page-locked already (all of it: by cudaHostAlloc or
                                cudaHostRegister, or because it is the host memory of another pool) is

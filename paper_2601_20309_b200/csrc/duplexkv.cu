@@ -15,7 +15,10 @@
 #include <cstdlib>
 #include <cstring>
 #include <new>
+#include <thread>
 #include <vector>
+
+#include <sys/mman.h>
 
 namespace {
 
@@ -133,6 +136,8 @@ struct kv_pool {
     uint8_t *host = nullptr;           // host address of the host pool
     uint8_t *host_dev = nullptr;       // the same memory as the device sees it
     bool owns_host = false, registered_host = false;
+    void *host_map = nullptr;           // anonymous mapping behind `host` when the library made it that way
+    size_t host_map_len = 0;
     int sm_count = 0;
     int64_t max_pitch = 0;             // largest row pitch a 2-D copy-engine transfer accepts
     DirState dir[2];                   // 0 = out, 1 = in
@@ -1160,6 +1165,67 @@ void harvest_call_timing(kv_pool *p)
     p->union_valid = p->union_synced = false;
 }
 
+// Host pool made by the library: an anonymous mapping, asked to be backed by transparent huge pages,
+// touched by several threads and then page-locked with cudaHostRegister.  Page-locking 120 GB this way
+// takes a fraction of what cudaHostAlloc takes for it (measured on 4 GiB: 0.6 s against 2.0 s, single
+// thread; the copy engines' rates are the same either way).  Returns nullptr when the mapping cannot be
+// made, when the system does not have that much memory available, or when CUDA refuses to register it;
+// the caller then falls back to cudaHostAlloc.
+int64_t mem_available_bytes()
+{
+    FILE *f = fopen("/proc/meminfo", "r");
+    if (!f) return -1;
+    char line[256];
+    long long kb = -1;
+    while (fgets(line, sizeof line, f))
+        if (sscanf(line, "MemAvailable: %lld kB", &kb) == 1) break;
+    fclose(f);
+    return kb < 0 ? -1 : (int64_t)kb * 1024;
+}
+
+uint8_t *map_host_pool(size_t bytes, void *&map, size_t &map_len)
+{
+    const char *how = getenv("DUPLEXKV_HOST_ALLOC");
+    if (how && strcmp(how, "cuda") == 0) return nullptr;
+    const int64_t avail = mem_available_bytes();
+    if (avail >= 0 && (double)bytes > 0.95 * (double)avail) return nullptr;   // never touch more than the box can give
+    const size_t huge = (size_t)2 << 20;
+    map_len = bytes + huge;
+    map = mmap(nullptr, map_len, PROT_READ | PROT_WRITE, MAP_PRIVATE | MAP_ANONYMOUS, -1, 0);
+    if (map == MAP_FAILED) {
+        map = nullptr;
+        return nullptr;
+    }
+    uint8_t *base = (uint8_t *)(((uintptr_t)map + huge - 1) & ~(uintptr_t)(huge - 1));
+    (void)madvise(base, bytes, MADV_HUGEPAGE);            // a hint: ordinary pages do as well, only slower to lock
+    // first touch, one byte per 4 KiB page, slices of whole huge pages per thread
+    unsigned threads = std::thread::hardware_concurrency();
+    threads = std::max(1u, std::min(threads, 16u));
+    if (bytes < ((size_t)256 << 20)) threads = 1;
+    const size_t pages = (bytes + huge - 1) / huge;
+    auto touch = [&](unsigned t) {
+        const size_t lo = pages * t / threads * huge, hi = std::min(bytes, pages * (t + 1) / threads * huge);
+        for (size_t o = lo; o < hi; o += 4096) ((volatile uint8_t *)base)[o] = 0;
+    };
+    try {
+        std::vector<std::thread> pool;
+        for (unsigned t = 1; t < threads; ++t) pool.emplace_back(touch, t);
+        touch(0);
+        for (auto &th : pool) th.join();
+    } catch (...) {
+        munmap(map, map_len);
+        map = nullptr;
+        return nullptr;
+    }
+    if (cudaHostRegister(base, bytes, cudaHostRegisterMapped | cudaHostRegisterPortable) != cudaSuccess) {
+        (void)cudaGetLastError();
+        munmap(map, map_len);
+        map = nullptr;
+        return nullptr;
+    }
+    return base;
+}
+
 }  // namespace
 
 // =================================================================================================
@@ -1300,6 +1366,8 @@ int32_t kv_pool_create(const kv_pool_config_t *cfg, kv_pool_t **out)
             }
             p->registered_host = true;
         }
+    } else if ((p->host = map_host_pool(host_bytes, p->host_map, p->host_map_len)) != nullptr) {
+        p->registered_host = true;      // unregistered and unmapped at destroy
     } else {
         cudaError_t e = cudaHostAlloc((void **)&p->host, host_bytes, cudaHostAllocMapped | cudaHostAllocPortable);
         if (e != cudaSuccess) {
@@ -1406,6 +1474,7 @@ int32_t kv_pool_destroy(kv_pool_t *p)
     if (p->status_host) (void)cudaFreeHost(p->status_host);
     if (p->owns_host && p->host) (void)cudaFreeHost(p->host);
     if (p->registered_host) (void)cudaHostUnregister(p->host);
+    if (p->host_map) (void)munmap(p->host_map, p->host_map_len);
     (void)cudaGetLastError();
     delete p;
     return KV_OK;
