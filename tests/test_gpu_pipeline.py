@@ -230,3 +230,32 @@ def test_second_pool_over_page_locked_memory_of_the_first():
         a.assert_equal("first pool after the second one is gone")
     finally:
         a.close()
+
+
+@pytest.mark.parametrize("how", ["cuda", None], ids=["cudaHostAlloc", "huge-page-mapping"])
+@pytest.mark.parametrize("path", [1, 2], ids=["zerocopy", "staged"])
+def test_both_ways_of_allocating_the_host_pool(how, path):
+    """The library's own host pool is a registered huge-page mapping by default and cudaHostAlloc memory on
+    DUPLEXKV_HOST_ALLOC=cuda (and whenever the mapping cannot be had): same results, and the pool's memory can
+    be written and read through kv_host_ptr either way.  300 MiB, so that several threads touch it."""
+    shape = W.KVShape(4, 16, 8, 128)                                              # 256 KiB blocks
+    nbg, nbh = 300, 1200
+    saved = os.environ.pop("DUPLEXKV_HOST_ALLOC", None)
+    try:
+        if how:
+            os.environ["DUPLEXKV_HOST_ALLOC"] = how
+        p = _pair(shape, nbg, nbh, seed=31, path=path)
+        try:
+            base, nbytes = p.pool.kv_host_ptr()
+            assert nbytes == nbh * shape.block_bytes and base % 4096 == 0
+            rng = np.random.default_rng(8)
+            pg, ph = rng.permutation(nbg).astype(np.int32), rng.permutation(nbh).astype(np.int32)
+            r = W.Rotation(pg[:140], ph[:140], ph[140:280], pg[140:280], np.zeros(1), np.zeros(1))
+            assert p.rotate_both(r) == 0
+            p.assert_equal(f"host pool allocated by {how or 'the default'}")
+        finally:
+            p.close()
+    finally:
+        os.environ.pop("DUPLEXKV_HOST_ALLOC", None)
+        if saved is not None:
+            os.environ["DUPLEXKV_HOST_ALLOC"] = saved
