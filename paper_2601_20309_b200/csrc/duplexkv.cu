@@ -1169,8 +1169,8 @@ void harvest_call_timing(kv_pool *p)
 // touched by several threads and then page-locked with cudaHostRegister.  Page-locking 120 GB this way
 // takes a fraction of what cudaHostAlloc takes for it (measured on 4 GiB: 0.6 s against 2.0 s, single
 // thread; the copy engines' rates are the same either way).  Returns nullptr when the mapping cannot be
-// made, when the system does not have that much memory available, or when CUDA refuses to register it;
-// the caller then falls back to cudaHostAlloc.
+// made, when the system (or the process's memory control group) does not have that much memory available, or
+// when CUDA refuses to register it; the caller then falls back to cudaHostAlloc.
 int64_t mem_available_bytes()
 {
     FILE *f = fopen("/proc/meminfo", "r");
@@ -1183,12 +1183,34 @@ int64_t mem_available_bytes()
     return kb < 0 ? -1 : (int64_t)kb * 1024;
 }
 
+// bytes this process may still take under its memory control group (v2, else v1), or -1 when there is no limit
+int64_t cgroup_headroom_bytes()
+{
+    auto read_ll = [](const char *path, long long &v) {
+        FILE *f = fopen(path, "r");
+        if (!f) return false;
+        char buf[64] = "";
+        const bool ok = fgets(buf, sizeof buf, f) != nullptr && sscanf(buf, "%lld", &v) == 1;   // "max" does not parse
+        fclose(f);
+        return ok;
+    };
+    long long limit = 0, used = 0;
+    if (read_ll("/sys/fs/cgroup/memory.max", limit) && read_ll("/sys/fs/cgroup/memory.current", used))
+        return std::max<long long>(0, limit - used);
+    if (read_ll("/sys/fs/cgroup/memory/memory.limit_in_bytes", limit) &&
+        read_ll("/sys/fs/cgroup/memory/memory.usage_in_bytes", used) && limit < (1ll << 60))
+        return std::max<long long>(0, limit - used);
+    return -1;
+}
+
 uint8_t *map_host_pool(size_t bytes, void *&map, size_t &map_len)
 {
     const char *how = getenv("DUPLEXKV_HOST_ALLOC");
     if (how && strcmp(how, "cuda") == 0) return nullptr;
-    const int64_t avail = mem_available_bytes();
-    if (avail >= 0 && (double)bytes > 0.95 * (double)avail) return nullptr;   // never touch more than the box can give
+    // never touch more than the box, or this process's control group, can give: touching is what takes the memory
+    const int64_t avail = mem_available_bytes(), room = cgroup_headroom_bytes();
+    if (avail >= 0 && (double)bytes > 0.95 * (double)avail) return nullptr;
+    if (room >= 0 && (double)bytes > 0.95 * (double)room) return nullptr;
     const size_t huge = (size_t)2 << 20;
     map_len = bytes + huge;
     map = mmap(nullptr, map_len, PROT_READ | PROT_WRITE, MAP_PRIVATE | MAP_ANONYMOUS, -1, 0);
