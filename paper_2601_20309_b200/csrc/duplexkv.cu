@@ -19,6 +19,8 @@
 #include <vector>
 
 #include <sys/mman.h>
+#include <sys/syscall.h>
+#include <unistd.h>
 
 namespace {
 
@@ -1203,7 +1205,34 @@ int64_t cgroup_headroom_bytes()
     return -1;
 }
 
-uint8_t *map_host_pool(size_t bytes, void *&map, size_t &map_len)
+// Ask the kernel to take the pages of [base, base + bytes) from the memory node the GPU hangs off, where
+// the box has more than one (the node is read from the GPU's PCI entry in sysfs): transfers to the other
+// socket's memory cross the sockets' interconnect.  A preference, not a binding; every failure is ignored.
+void prefer_memory_node_of_gpu(void *base, size_t bytes, int device_id)
+{
+    char bdf[32] = "";
+    if (cudaDeviceGetPCIBusId(bdf, (int)sizeof bdf, device_id) != cudaSuccess) {
+        (void)cudaGetLastError();
+        return;
+    }
+    for (char *c = bdf; *c; ++c)
+        if (*c >= 'A' && *c <= 'F') *c = (char)(*c - 'A' + 'a');
+    char path[96];
+    snprintf(path, sizeof path, "/sys/bus/pci/devices/%s/numa_node", bdf);
+    FILE *f = fopen(path, "r");
+    if (!f) return;
+    int node = -1;
+    const bool ok = fscanf(f, "%d", &node) == 1;
+    fclose(f);
+    if (!ok || node < 0 || node >= 1024) return;
+    unsigned long mask[1024 / (8 * sizeof(unsigned long))] = {};
+    mask[(size_t)node / (8 * sizeof(unsigned long))] |= 1ul << ((size_t)node % (8 * sizeof(unsigned long)));
+#ifdef SYS_mbind
+    (void)syscall(SYS_mbind, base, bytes, 1 /* MPOL_PREFERRED */, mask, 1024ul + 1, 0u);
+#endif
+}
+
+uint8_t *map_host_pool(size_t bytes, int device_id, void *&map, size_t &map_len)
 {
     const char *how = getenv("DUPLEXKV_HOST_ALLOC");
     if (how && strcmp(how, "cuda") == 0) return nullptr;
@@ -1220,6 +1249,7 @@ uint8_t *map_host_pool(size_t bytes, void *&map, size_t &map_len)
     }
     uint8_t *base = (uint8_t *)(((uintptr_t)map + huge - 1) & ~(uintptr_t)(huge - 1));
     (void)madvise(base, bytes, MADV_HUGEPAGE);            // a hint: ordinary pages do as well, only slower to lock
+    prefer_memory_node_of_gpu(base, bytes, device_id);
     // first touch, one byte per 4 KiB page, slices of whole huge pages per thread
     unsigned threads = std::thread::hardware_concurrency();
     threads = std::max(1u, std::min(threads, 16u));
@@ -1388,7 +1418,7 @@ int32_t kv_pool_create(const kv_pool_config_t *cfg, kv_pool_t **out)
             }
             p->registered_host = true;
         }
-    } else if ((p->host = map_host_pool(host_bytes, p->host_map, p->host_map_len)) != nullptr) {
+    } else if ((p->host = map_host_pool(host_bytes, cfg->device_id, p->host_map, p->host_map_len)) != nullptr) {
         p->registered_host = true;      // unregistered and unmapped at destroy
     } else {
         cudaError_t e = cudaHostAlloc((void **)&p->host, host_bytes, cudaHostAllocMapped | cudaHostAllocPortable);
