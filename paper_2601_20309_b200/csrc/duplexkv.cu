@@ -1249,6 +1249,7 @@ uint8_t *map_host_pool(size_t bytes, int device_id, void *&map, size_t &map_len)
     }
     uint8_t *base = (uint8_t *)(((uintptr_t)map + huge - 1) & ~(uintptr_t)(huge - 1));
     (void)madvise(base, bytes, MADV_HUGEPAGE);            // a hint: ordinary pages do as well, only slower to lock
+    (void)madvise(base, bytes, MADV_DONTFORK);            // a forked child must not share (and copy-on-write) pages the GPU writes
     prefer_memory_node_of_gpu(base, bytes, device_id);
     // first touch, one byte per 4 KiB page, slices of whole huge pages per thread
     unsigned threads = std::thread::hardware_concurrency();
