@@ -58,7 +58,7 @@ extern "C" {
 #define KV_DEV_BLOCK_FIRST    1     /* [block][layer][K|V]...: the paper's redesigned storage order      */
 
 /* transfer paths (how the host link is driven) */
-#define KV_PATH_AUTO          0     /* per call.  8 MiB or less per direction (2 MiB for blocks under 2 MiB):
+#define KV_PATH_AUTO          0     /* per call.  8 MiB or less per direction (blocks under 2 MiB: two blocks at most):
                                        CE2D, the lowest fixed cost.  Larger calls: STAGED when the
                                        copy-engine transfers the call needs would average 2.5 MiB or more,
                                        else ZEROCOPY (see kv_path_for)                                   */

@@ -32,10 +32,13 @@ constexpr int64_t KV_AUTO_MIN_TRANSFER = 5ll << 19;   // AUTO: staged when its t
 // 212 us for 1 / 2 / 4 blocks each way against 85 / 141 / 231 us staged and 87 / 143 / 247 us for the
 // zero-copy kernels); from 16 MiB on the staged path (one chunk, ids in the launch parameters, four-block
 // lattices) is ahead (406 / 789 us at 8 / 16 blocks against 451 / 847 and 463 / 908) and the transfer-size
-// rule decides.  With 1 MiB blocks one transfer per block wins only up to 2 MiB (44 / 75 us for 1 / 2
-// blocks); above that the transfer-size rule picks the zero-copy kernels, which lead up to ~128 MiB.
+// rule decides.  With smaller blocks one transfer per block wins only for one or two blocks per direction
+// (1 MiB blocks: 44 / 70 us for 1 / 2 blocks against 59 / 90 zero-copy, but 161 against 144 for 4; 256 KiB
+// blocks: 28 / 43-48 against 43 / 43, but 69 / 122 against 60 / 90 for 4 / 8); above that the transfer-size
+// rule picks the zero-copy kernels, which lead up to ~128 MiB.
 constexpr int64_t KV_AUTO_TINY_BYTES = 8ll << 20;
 constexpr int64_t KV_AUTO_TINY_BYTES_SMALL_BLOCKS = 2ll << 20;
+constexpr int64_t KV_AUTO_TINY_COUNT_SMALL_BLOCKS = 2;
 constexpr int64_t KV_MERGE_MIN_MEAN_RUN = 8;
 constexpr int64_t KV_QUAD_MAX_GAP = 256;              // STAGED, scattered ids: largest row gap (blocks) of a four-block lattice
 constexpr int64_t KV_QUAD_ENOUGH_BYTES = 8ll << 20;  //         no lattices when a pair of blocks already carries this much
@@ -1043,8 +1046,8 @@ int32_t run_calls(kv_pool *p, DirCall *calls, int ncalls, const bool *wait_other
             const DirState &o = p->dir[1 - calls[k].d];
             wait_ev[k] = o.ev_end[o.issued % KV_SLOTS];
         }
-    // KV_PATH_AUTO is settled per call.  A call that moves very little (KV_AUTO_TINY_BYTES per direction, less
-    // for blocks under 2 MiB) is all fixed cost and goes as one copy-engine transfer per block.  Otherwise the
+    // KV_PATH_AUTO is settled per call.  A call that moves very little (KV_AUTO_TINY_BYTES per direction; for
+    // blocks under 2 MiB at most two blocks and 2 MiB) is all fixed cost and goes as one copy-engine transfer per block.  Otherwise the
     // staged transfers are planned first (cheap: a sort of the ids and one sweep over them) and the staged
     // path is taken when its transfers would carry KV_AUTO_MIN_TRANSFER bytes or more on average, the
     // zero-copy kernels when not.  Both directions of a rotate take the same path (a kernel on one direction
@@ -1055,8 +1058,11 @@ int32_t run_calls(kv_pool *p, DirCall *calls, int ncalls, const bool *wait_other
             calls[k].path = p->dir[calls[k].d].path;
             if (calls[k].path == KV_PATH_AUTO) largest = std::max(largest, calls[k].n * p->blk);
         }
+        const bool tiny = p->blk >= (2ll << 20)
+                              ? largest <= KV_AUTO_TINY_BYTES
+                              : largest <= KV_AUTO_TINY_BYTES_SMALL_BLOCKS && largest <= KV_AUTO_TINY_COUNT_SMALL_BLOCKS * p->blk;
         int chosen;
-        if (largest <= (p->blk >= (2ll << 20) ? KV_AUTO_TINY_BYTES : KV_AUTO_TINY_BYTES_SMALL_BLOCKS)) {
+        if (tiny) {
             chosen = KV_PATH_CE2D;
         } else {
             int64_t bytes = 0, ops = 0;

@@ -299,11 +299,11 @@ def overlap(out) -> None:
               f"{r['compute_beside_rotate_tbs']} | {r['compute_slowdown_pct_while_rotating']} % | {r['rotate_slowdown_pct']} % |")
 
 
-def latency(out, block_size: int = 16) -> None:
+def latency(out, block_size: int = 16, kv_heads: int = 8) -> None:
     import time
     import numpy as np
     import torch
-    shape = W.KVShape(32, block_size)
+    shape = W.KVShape(32, block_size, kv_heads)
     nb = 4096 * 16 // block_size if block_size < 16 else 4096
     dev = torch.empty(nb * shape.block_bytes, dtype=torch.uint8, device="cuda:0")
     pool = B.KVPool(shape.num_layers, shape.block_size, shape.kv_heads, shape.head_dim, nb, nb, dev.data_ptr())
@@ -604,7 +604,7 @@ def main() -> None:
                     help="paths: device pool layout (block-first = the paper's redesigned storage order)")
     ap.add_argument("--pool-gib", type=int, default=4, help="segments: device pool size in GiB")
     ap.add_argument("--kv-heads", type=int, default=8,
-                    help="paths: KV heads held by this GPU (8 = the whole 8B shape; 1, 2 or 4 = one rank's shard under tensor parallelism)")
+                    help="paths, latency: KV heads held by this GPU (8 = the whole 8B shape; 1, 2 or 4 = one rank's shard under tensor parallelism)")
     a = ap.parse_args()
     import torch
     if not torch.cuda.is_available():
@@ -619,7 +619,7 @@ def main() -> None:
     elif a.what == "overlap":
         overlap(out)
     elif a.what == "latency":
-        latency(out, a.block_size)
+        latency(out, a.block_size, a.kv_heads)
     elif a.what == "handoff":
         handoff(out)
     elif a.what == "lvf":
